@@ -1,0 +1,138 @@
+// Shared host/device helpers of the AirCache sm_100a library: error plumbing, the workspace
+// carve-up, argument checks and a few device intrinsics.  Nothing in here is used by the CPU oracle.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/aircache.h"
+
+namespace aircache {
+
+constexpr int kMaxWindow = 64;
+constexpr int kMaxGroup = 16;         // query heads per KV head
+constexpr int kMaxRegions = 2048;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
+constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)
+constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ---------------------------------------------------------------------------------------------
+// error plumbing
+// ---------------------------------------------------------------------------------------------
+void set_last_cuda_error(cudaError_t e);
+
+#define AIRCACHE_CUDA_TRY(expr)                         \
+    do {                                                \
+        cudaError_t _e = (expr);                        \
+        if (_e != cudaSuccess) {                        \
+            ::aircache::set_last_cuda_error(_e);        \
+            return AIRCACHE_ERR_CUDA;                   \
+        }                                               \
+    } while (0)
+
+#define AIRCACHE_LAUNCH_CHECK()                         \
+    do {                                                \
+        cudaError_t _e = cudaGetLastError();            \
+        if (_e != cudaSuccess) {                        \
+            ::aircache::set_last_cuda_error(_e);        \
+            return AIRCACHE_ERR_CUDA;                   \
+        }                                               \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// shape helpers and the workspace carve-up (host arithmetic)
+// ---------------------------------------------------------------------------------------------
+int check_shape(const aircache_shape_t *s);
+int check_full(const aircache_shape_t *s, const aircache_full_t *f);
+int64_t kept_per_sequence(const aircache_shape_t *s, double ratio);
+
+inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Elite rows one KV group can have at most, padded to the MMA tile of 8 rows.
+inline int score_row_cap(const aircache_shape_t *s) {
+    int g = s->n_q_heads / s->n_kv_heads;
+    return (int)align_up((int64_t)g * s->window, 16);
+}
+
+// Visual-key chunks of the statistics pass: enough CTAs for about four waves on a B200,
+// at least 256 keys per chunk.  A function of the shape only, so results are reproducible.
+inline int score_chunks(const aircache_shape_t *s) {
+    int64_t groups = (int64_t)s->n_layers * s->batch * s->n_kv_heads;
+    int64_t want = (592 + groups - 1) / groups;
+    int64_t most = (s->n_visual + 255) / 256;
+    if (want > most) want = most;
+    if (want < 1) want = 1;
+    return (int)want;
+}
+
+struct WsLayout {
+    int64_t status;       // u32 status word (256 bytes reserved)
+    int64_t row_count;    // i32  [L*B*Hkv]            elite rows of the KV group
+    int64_t row_info;     // i32  [L*B*Hkv][cap]       (head within group << 8) | window slot
+    int64_t row_coef;     // f32  [L*B*Hkv][cap]       1 / (|E_h| * Hq)
+    int64_t row_text;     // f32x2[L*B*Hkv][cap]       (max, sum) of the visible elite text logits, log2 domain
+    int64_t chunk_stats;  // f32x2[L*B*Hkv][chunks][cap]  (max, sum) over one chunk of visual keys
+    int64_t mom_strength; // f64  [L*B]
+    int64_t mom_skew;     // f64  [L*B]
+    int64_t alloc_w;      // f64  [L*B]
+    int64_t alloc_share;  // f64  [L*B]
+    int64_t alloc_active; // i32  [L*B]
+    int64_t kept;         // i32  [L*B*Nv]             kept-token lists when the caller passes none
+    int64_t plan;         // i32  [L*B + 2]            unit prefix of the decode schedule (+ total)
+    int64_t partials;     // f32  [2*kMaxDecodeCtas][Hq*(d+2)]
+    int64_t total;
+};
+
+WsLayout ws_layout(const aircache_shape_t *s);
+
+template <typename T>
+inline T *ws_ptr(void *ws, int64_t off) {
+    return reinterpret_cast<T *>(reinterpret_cast<char *>(ws) + off);
+}
+
+// entry points implemented per translation unit
+int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void *q_window, float alpha,
+                 float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st);
+int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, int32_t mode, int32_t *budgets,
+                  double *strength, double *skewness, aircache_ragged_t *layout, void *ws, cudaStream_t st);
+int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const float *scores,
+                   const int32_t *budgets, double ratio, aircache_ragged_t *out, int32_t *kept_idx, void *ws,
+                   cudaStream_t st);
+int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out, void *ws,
+                  cudaStream_t st);
+int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,
+                  int32_t appended, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ float bf16lo(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
+__device__ __forceinline__ float bf16_to_f32(uint16_t h) { return __uint_as_float((uint32_t)h << 16); }
+
+// D += A(16x16, bf16, row) * B(16x8, bf16, col), fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Merge two (max, sum-of-exp2) pairs of the same softmax row.
+__device__ __forceinline__ void merge_stats(float &m, float &z, float m2, float z2) {
+    float mn = fmaxf(m, m2);
+    z = z * fast_exp2(m - mn) + z2 * fast_exp2(m2 - mn);
+    m = mn;
+}
+#endif
+
+}  // namespace aircache

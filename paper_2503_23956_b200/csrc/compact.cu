@@ -1,0 +1,270 @@
+// aircache_compact: per-region top-k of the importance scores and the gather that packs the kept
+// visual rows and all text rows into the ragged cache (Algorithm 1, second loop); aircache_append (Eq. 2).
+//
+//   select_kernel  one CTA per region.  Radix select, most significant byte first, on an order-preserving
+//                  integer image of the fp32 score: four 256-bin histogram passes find the value of the
+//                  k-th largest score and how many of its duplicates are needed; one ordered pass then
+//                  emits the kept token indices in ascending order, duplicates of the threshold value
+//                  taken from the lowest indices.
+//   gather_kernel  one warp per output row [Hkv, d] of K' and of V': 16-byte loads along the source row's
+//                  head slices, 16-byte stores to the packed row.  Region of a row by binary search in the
+//                  offsets table.
+#include "common.cuh"
+
+namespace aircache {
+
+namespace {
+
+constexpr int kSelThreads = 512;
+constexpr int kSelSmemKeys = 40960;  // scores kept in shared memory up to this many visual tokens
+
+__device__ __forceinline__ uint32_t order_key(float x) {
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive block scan of one int per thread; returns the exclusive prefix, total in *total.
+__device__ __forceinline__ int block_excl_scan(int v, int *s_warp, int *total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int sh = 1; sh < 32; sh <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+        if (lane >= sh) incl += o;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < (kSelThreads / 32) ? s_warp[lane] : 0;
+#pragma unroll
+        for (int sh = 1; sh < 32; sh <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, w, sh);
+            if (lane >= sh) w += o;
+        }
+        if (lane < kSelThreads / 32) s_warp[lane] = w;
+    }
+    __syncthreads();
+    *total = s_warp[kSelThreads / 32 - 1];
+    return incl - v + (warp > 0 ? s_warp[warp - 1] : 0);
+}
+
+template <bool SMEM_KEYS>
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__restrict__ scores,
+                                                             const int32_t *__restrict__ budgets,
+                                                             const int64_t *__restrict__ offsets, int n_visual,
+                                                             int n_text, int slack, int32_t *__restrict__ kept) {
+    extern __shared__ uint32_t s_keys[];
+    __shared__ int s_hist[256];
+    __shared__ int s_warp[kSelThreads / 32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+
+    const int r = blockIdx.x;
+    const int k = budgets[r];
+    int32_t *out = kept + (offsets[r] - (int64_t)r * (n_text + slack));
+    const float *x = scores + (int64_t)r * n_visual;
+    if (k <= 0) return;
+    if (k >= n_visual) {
+        for (int i = threadIdx.x; i < n_visual; i += kSelThreads) out[i] = i;
+        return;
+    }
+    if (SMEM_KEYS) {
+        for (int i = threadIdx.x; i < n_visual; i += kSelThreads) s_keys[i] = order_key(x[i]);
+    }
+    auto key_at = [&](int i) -> uint32_t { return SMEM_KEYS ? s_keys[i] : order_key(x[i]); };
+
+    if (threadIdx.x == 0) { s_prefix = 0; s_remaining = k; }
+    uint32_t mask = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += kSelThreads) s_hist[i] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int i = threadIdx.x; i < n_visual; i += kSelThreads) {
+            const uint32_t key = key_at(i);
+            if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            // warp 0: walk the bins from the largest digit down until `remaining` keys are covered
+            const int lane = threadIdx.x;
+            int remaining = s_remaining;
+            int chosen = -1;
+            for (int base = 224; base >= 0 && chosen < 0; base -= 32) {
+                const int bin = base + 31 - lane;  // lane 0 holds the largest digit of the group
+                const int c = s_hist[bin];
+                int incl = c;
+#pragma unroll
+                for (int sh = 1; sh < 32; sh <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+                    if (lane >= sh) incl += o;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, incl >= remaining);
+                if (hit) {
+                    const int src = __ffs(hit) - 1;
+                    const int before = __shfl_sync(0xffffffffu, incl - c, src);
+                    chosen = base + 31 - src;
+                    remaining -= before;
+                } else {
+                    remaining -= __shfl_sync(0xffffffffu, incl, 31);
+                }
+            }
+            if (lane == 0) {
+                s_prefix = prefix | ((uint32_t)chosen << shift);
+                s_remaining = remaining;
+            }
+        }
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    const uint32_t thr = s_prefix;   // image of the k-th largest score
+    const int need_eq = s_remaining; // how many tokens equal to it are kept (lowest indices first)
+
+    // ordered emit: thread t owns the contiguous index range [i0, i1)
+    const int per = (n_visual + kSelThreads - 1) / kSelThreads;
+    const int i0 = min(n_visual, (int)threadIdx.x * per), i1 = min(n_visual, i0 + per);
+    int n_eq = 0, n_gt = 0;
+    for (int i = i0; i < i1; ++i) {
+        const uint32_t key = key_at(i);
+        n_eq += key == thr;
+        n_gt += key > thr;
+    }
+    int tot;
+    const int eq_before = block_excl_scan(n_eq, s_warp, &tot);
+    int take_eq = min(max(need_eq - eq_before, 0), n_eq);
+    const int pos0 = block_excl_scan(n_gt + take_eq, s_warp, &tot);
+    int pos = pos0;
+    for (int i = i0; i < i1; ++i) {
+        const uint32_t key = key_at(i);
+        bool keep = key > thr;
+        if (key == thr && take_eq > 0) { keep = true; --take_eq; }
+        if (keep) out[pos++] = i;
+    }
+}
+
+struct GatherParams {
+    const uint16_t *k, *v;
+    int64_t s_layer, s_batch, s_head, s_token;
+    uint16_t *k_out, *v_out;
+    const int64_t *offsets;
+    const int32_t *lens;
+    const int32_t *budgets;
+    const int32_t *kept;
+    int64_t rows_cap;  // rows covered by the launch
+    int L, B, Hkv, d, Nv, Nt, slack;
+};
+
+constexpr int kGatherThreads = 256;
+constexpr int kGatherRowsPerWarp = 4;
+
+__global__ void __launch_bounds__(kGatherThreads) gather_kernel(GatherParams p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
+    const int n_regions = p.L * p.B;
+    const int64_t total = p.offsets[n_regions];
+    const int vec_per_head = p.d / 8;             // 16-byte vectors per head slice
+    const int vec_per_row = p.Hkv * vec_per_head;
+
+    int64_t src_off[kGatherRowsPerWarp];
+    int64_t dst_row[kGatherRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+        const int64_t row = warp_global * kGatherRowsPerWarp + i;
+        dst_row[i] = -1;
+        src_off[i] = 0;
+        if (row >= total) continue;
+        // region r with offsets[r] <= row < offsets[r+1]
+        int lo = 0, hi = n_regions - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (p.offsets[mid] <= row) lo = mid; else hi = mid - 1;
+        }
+        const int r = lo;
+        const int64_t base = p.offsets[r];
+        const int j = (int)(row - base);
+        if (j >= p.lens[r]) continue;  // slack row
+        const int n = p.budgets[r];
+        const int l = r / p.B, b = r % p.B;
+        const int tok = j < n ? p.kept[base - (int64_t)r * (p.Nt + p.slack) + j] : p.Nv + (j - n);
+        src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)tok * p.s_token;
+        dst_row[i] = row;
+    }
+    for (int v0 = lane; v0 < vec_per_row; v0 += 32) {
+        const int g = v0 / vec_per_head, c = v0 % vec_per_head;
+        uint4 kk[kGatherRowsPerWarp], vv[kGatherRowsPerWarp];
+#pragma unroll
+        for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+            if (dst_row[i] < 0) continue;
+            const int64_t so = src_off[i] + (int64_t)g * p.s_head + c * 8;
+            kk[i] = __ldg(reinterpret_cast<const uint4 *>(p.k + so));
+            vv[i] = __ldg(reinterpret_cast<const uint4 *>(p.v + so));
+        }
+#pragma unroll
+        for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+            if (dst_row[i] < 0) continue;
+            const int64_t dof = (dst_row[i] * p.Hkv + g) * p.d + c * 8;
+            *reinterpret_cast<uint4 *>(p.k_out + dof) = kk[i];
+            *reinterpret_cast<uint4 *>(p.v_out + dof) = vv[i];
+        }
+    }
+}
+
+__global__ void append_kernel(uint16_t *k_out, uint16_t *v_out, const int64_t *offsets, int32_t *lens,
+                              const uint16_t *k_new, const uint16_t *v_new, int row_elems) {
+    const int r = blockIdx.x;
+    const int64_t dst = (offsets[r] + lens[r]) * row_elems;
+    const int64_t src = (int64_t)r * row_elems;
+    for (int c = threadIdx.x * 8; c < row_elems; c += blockDim.x * 8) {
+        *reinterpret_cast<uint4 *>(k_out + dst + c) = *reinterpret_cast<const uint4 *>(k_new + src + c);
+        *reinterpret_cast<uint4 *>(v_out + dst + c) = *reinterpret_cast<const uint4 *>(v_new + src + c);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) lens[r] += 1;
+}
+
+}  // namespace
+
+int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const float *scores,
+                   const int32_t *budgets, double ratio, aircache_ragged_t *out, int32_t *kept_idx, void *ws,
+                   cudaStream_t st) {
+    const WsLayout w = ws_layout(s);
+    const int LB = s->n_layers * s->batch;
+    int32_t *kept = kept_idx ? kept_idx : ws_ptr<int32_t>(ws, w.kept);
+    if (s->n_visual <= kSelSmemKeys) {
+        const size_t smem = (size_t)s->n_visual * 4;
+        AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               kSelSmemKeys * 4));
+        select_kernel<true><<<LB, kSelThreads, smem, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
+                                                           s->slack, kept);
+    } else {
+        select_kernel<false><<<LB, kSelThreads, 0, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
+                                                         s->slack, kept);
+    }
+    AIRCACHE_LAUNCH_CHECK();
+
+    GatherParams p;
+    p.k = (const uint16_t *)f->k; p.v = (const uint16_t *)f->v;
+    p.s_layer = f->stride_layer; p.s_batch = f->stride_batch; p.s_head = f->stride_head; p.s_token = f->stride_token;
+    p.k_out = (uint16_t *)out->k; p.v_out = (uint16_t *)out->v;
+    p.offsets = out->offsets; p.lens = out->lens; p.budgets = budgets; p.kept = kept;
+    p.rows_cap = (int64_t)s->batch * (kept_per_sequence(s, ratio) + (int64_t)s->n_layers * (s->n_text + s->slack));
+    p.L = s->n_layers; p.B = s->batch; p.Hkv = s->n_kv_heads; p.d = s->head_dim;
+    p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack;
+    const int64_t rows_per_block = (kGatherThreads / 32) * kGatherRowsPerWarp;
+    const int64_t blocks = (p.rows_cap + rows_per_block - 1) / rows_per_block;
+    gather_kernel<<<(unsigned)blocks, kGatherThreads, 0, st>>>(p);
+    AIRCACHE_LAUNCH_CHECK();
+    return AIRCACHE_OK;
+}
+
+int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,
+                  int32_t appended, cudaStream_t st) {
+    (void)appended;
+    append_kernel<<<s->n_layers * s->batch, 64, 0, st>>>((uint16_t *)c->k, (uint16_t *)c->v, c->offsets, c->lens,
+                                                         (const uint16_t *)k_new, (const uint16_t *)v_new,
+                                                         s->n_kv_heads * s->head_dim);
+    AIRCACHE_LAUNCH_CHECK();
+    return AIRCACHE_OK;
+}
+
+}  // namespace aircache

@@ -1,0 +1,586 @@
+// aircache_decode_attn: single-token attention over the ragged compressed cache (Section 3.1, token
+// decoding), all layers and sequences in one persistent launch plus a small combine launch.
+//
+// Work decomposition.  A "unit" is CH consecutive rows of one region (all KV heads, K and V).  Region r
+// has ceil(lens[r] / CH) units; every CTA first scans these counts into a prefix P (shared memory), then
+// takes the contiguous unit range [c * upc, (c+1) * upc) of the global unit list, upc = ceil(total / CTAs).
+// The load is therefore balanced to one unit regardless of how ragged the regions are.  Consecutive units
+// of one region accumulate in registers; a region that lies wholly inside one CTA's range is finished and
+// written by that CTA, otherwise the CTA writes an unnormalised partial (running max, sum, accumulator) and
+// combine_kernel merges the partials of the region in CTA order (split-K, fixed order).
+//
+// Inside a CTA.  One producer warp streams units through a ring of shared-memory stages with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle, one box of CH rows x 64 channels per KV head and half of
+// head_dim) and mbarriers.  Consumer warp (g, ks) owns KV head g and the 16-row block ks of every unit:
+//   S = Q_g K^T   mma.m16n8k16: the G query heads of the group are the M rows (padded to 16), keys are N;
+//                 K fragments come from ldmatrix on the swizzled tile
+//   online softmax in the exp2 domain, warp-shuffle row maxima over the quad that shares a row
+//   O += P V      P rounded to bf16 (the row sum uses the same rounded values), V fragments from
+//                 ldmatrix.trans
+// The G-fold reuse of every K/V row across the query heads of a group is what puts this on the tensor
+// pipe: with plain FMAs the kernel would need about 7 flop per byte, more than half of the fp32 peak at
+// full HBM rate.
+//
+// Every mbarrier wait is bounded: after kSpinLimit polls the waiter records a status word in the
+// workspace, raises a CTA-wide abort flag and the kernel drains and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace aircache {
+
+namespace {
+
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct DecodeParams {
+    const uint16_t *q;       // [L*B, Hq, D]
+    float *out;              // [L*B, Hq, D]
+    const int64_t *offsets;  // [L*B + 1]
+    const int32_t *lens;     // [L*B]
+    int32_t *plan;           // [L*B + 2] unit prefix written by CTA 0 for the combine kernel
+    float *partials;         // [2 * CTAs][Hq * (D + 2)]
+    uint32_t *status;
+    int n_regions, Hq, G;
+    float sl2;               // scale * log2(e)
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the wait gave up or another thread of the CTA already did.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                          uint32_t code) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (i > 64) __nanosleep(40);
+    }
+    atomicExch(status, code);
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void consumer_bar(int n_threads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory");
+}
+__device__ __forceinline__ float exp2_or_zero(float m, float m_new) {
+    return m == -INFINITY ? 0.f : fast_exp2(m - m_new);
+}
+
+template <int D, int HKV, bool G_HI>
+struct DecodeCfg {
+    static constexpr int NROW = G_HI ? 2 : 1;        // accumulator row groups in use (heads 0-7, heads 8-15)
+    static constexpr int NSTAGE = G_HI ? 2 : 3;      // ring depth (the wider merge buffer costs one stage)
+    static constexpr int KSPLIT = (8 / HKV) > 4 ? 4 : (8 / HKV);
+    static constexpr int CH = 16 * KSPLIT;           // rows per unit
+    static constexpr int NCW = HKV * KSPLIT;         // consumer warps
+    static constexpr int THREADS = (NCW + 1) * 32;
+    static constexpr int HALVES = D / 64;
+    static constexpr int SUBTILE = CH * 128;         // bytes of one (head, half) box
+    static constexpr int KV_BYTES = HKV * HALVES * SUBTILE;
+    static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+    // merge buffer: one slot per consumer warp with ks > 0
+    static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 2));
+    static constexpr int MERGE_BYTES = HKV * (KSPLIT - 1) * MERGE_FLOATS_PER_WARP * 4;
+    static constexpr int PLAN_BYTES = (kMaxRegions + 2) * 4;
+    static constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + MERGE_BYTES + PLAN_BYTES + 256;
+};
+
+// largest r with P[r] <= u (P non-decreasing, P[0] = 0, u < P[n])
+__device__ __forceinline__ int find_region(const int *P, int n, int u) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (P[mid] <= u) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+template <int D, int HKV, bool G_HI>
+__global__ void __launch_bounds__(DecodeCfg<D, HKV, G_HI>::THREADS, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, DecodeParams p) {
+    using C = DecodeCfg<D, HKV, G_HI>;
+    constexpr int KSPLIT = C::KSPLIT, CH = C::CH, NCW = C::NCW, NROW = C::NROW, kStages = C::NSTAGE;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *s_stage = smem;
+    float *s_merge = reinterpret_cast<float *>(smem + kStages * C::STAGE_BYTES);
+    int *s_P = reinterpret_cast<int *>(smem + kStages * C::STAGE_BYTES + C::MERGE_BYTES);
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + kStages * C::STAGE_BYTES + C::MERGE_BYTES + C::PLAN_BYTES);
+    __shared__ int s_part[C::THREADS];
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+    const int n = p.n_regions;
+
+    // ---- unit prefix of all regions (every CTA computes the same table) ----
+    {
+        const int per = (n + C::THREADS - 1) / C::THREADS;
+        const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
+        int local = 0;
+        for (int i = i0; i < i1; ++i) local += (max(p.lens[i], 0) + CH - 1) / CH;
+        s_part[tid] = local;
+        if (tid == 0) s_abort = 0;
+        __syncthreads();
+        if (wid == 0) {
+            // warp 0 turns s_part into an exclusive prefix
+            constexpr int PER_LANE = (C::THREADS + 31) / 32;
+            int sum = 0;
+            for (int j = 0; j < PER_LANE; ++j) {
+                const int idx = lane * PER_LANE + j;
+                if (idx < C::THREADS) sum += s_part[idx];
+            }
+            int incl = sum;
+#pragma unroll
+            for (int sh = 1; sh < 32; sh <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+                if (lane >= sh) incl += o;
+            }
+            int run = incl - sum;
+            for (int j = 0; j < PER_LANE; ++j) {
+                const int idx = lane * PER_LANE + j;
+                if (idx < C::THREADS) { const int v = s_part[idx]; s_part[idx] = run; run += v; }
+            }
+        }
+        __syncthreads();
+        int run = s_part[tid];
+        for (int i = i0; i < i1; ++i) {
+            s_P[i] = run;
+            run += (max(p.lens[i], 0) + CH - 1) / CH;
+        }
+        if (i1 == n && i0 < n) s_P[n] = run;
+        if (n == 0 && tid == 0) s_P[0] = 0;
+        if (tid == 0) {
+            for (int s = 0; s < kStages; ++s) {
+                mbar_init(smem_u32(&s_bar[s]), 1);             // full: the producer's expect_tx arrival
+                mbar_init(smem_u32(&s_bar[kStages + s]), NCW);  // empty: one arrival per consumer warp
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncthreads();
+    }
+    const int total = s_P[n];
+    if (blockIdx.x == 0) {
+        for (int i = tid; i <= n; i += C::THREADS) p.plan[i] = s_P[i];
+    }
+    const int upc = max(1, (total + (int)gridDim.x - 1) / (int)gridDim.x);
+    const int u0 = min(total, (int)blockIdx.x * upc), u1 = min(total, u0 + upc);
+    if (u0 >= u1) return;
+
+    if (wid == NCW) {
+        // =============================== producer warp ===============================
+        if (lane == 0) {
+            int r = find_region(s_P, n, u0);
+            int64_t row_base = p.offsets[r];
+            int it = 0;
+            bool ok = true;
+            for (int u = u0; u < u1 && ok; ++u, ++it) {
+                if (u >= s_P[r + 1]) {
+                    while (u >= s_P[r + 1]) ++r;
+                    row_base = p.offsets[r];
+                }
+                const int s = it % kStages;
+                if (it >= kStages)
+                    ok = mbar_wait(smem_u32(&s_bar[kStages + s]), ((it / kStages) & 1) ^ 1, &s_abort, p.status, 1);
+                if (!ok) break;
+                const int row0 = (int)(row_base + (int64_t)(u - s_P[r]) * CH);
+                const uint32_t full = smem_u32(&s_bar[s]);
+                mbar_expect_tx(full, C::STAGE_BYTES);
+                const uint32_t dst = smem_u32(s_stage + s * C::STAGE_BYTES);
+#pragma unroll
+                for (int g = 0; g < HKV; ++g) {
+#pragma unroll
+                    for (int hf = 0; hf < C::HALVES; ++hf) {
+                        const uint32_t off = (g * C::HALVES + hf) * C::SUBTILE;
+                        tma_load_3d(dst + off, &tm_k, hf * 64, g, row0, full);
+                        tma_load_3d(dst + C::KV_BYTES + off, &tm_v, hf * 64, g, row0, full);
+                    }
+                }
+            }
+            if (!ok) {
+                // drain: wait (bounded) for the loads already in flight before the CTA may exit
+                for (int j = max(0, it - kStages); j < it; ++j) {
+                    const uint32_t bar = smem_u32(&s_bar[j % kStages]);
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_test(bar, (j / kStages) & 1); ++i) __nanosleep(40);
+                }
+            }
+        }
+        return;
+    }
+
+    // ================================= consumer warps =================================
+    const int g = wid / KSPLIT, ks = wid % KSPLIT;
+    const int gid = lane >> 2, t = lane & 3;
+    const int G = p.G;
+
+    uint32_t qa[D / 16][4];
+    float oacc[D / 8][4];
+    float m_run[2], l_run[2];
+
+    auto load_q = [&](int r) {
+        const uint16_t *q_lo = p.q + ((int64_t)r * p.Hq + g * G + gid) * D;
+        const uint16_t *q_hi = q_lo + 8 * D;
+        const bool v_lo = gid < G, v_hi = G_HI && (gid + 8 < G);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+            qa[kk][0] = v_lo ? __ldg(reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 2 * t)) : 0u;
+            qa[kk][2] = v_lo ? __ldg(reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8 + 2 * t)) : 0u;
+            qa[kk][1] = v_hi ? __ldg(reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 2 * t)) : 0u;
+            qa[kk][3] = v_hi ? __ldg(reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8 + 2 * t)) : 0u;
+        }
+#pragma unroll
+        for (int nd = 0; nd < D / 8; ++nd) oacc[nd][0] = oacc[nd][1] = oacc[nd][2] = oacc[nd][3] = 0.f;
+        m_run[0] = m_run[1] = -INFINITY;
+        l_run[0] = l_run[1] = 0.f;
+    };
+
+    // Writes the region's result (whole region inside this CTA) or an unnormalised partial.
+    auto flush = [&](int r, int ustart, int uend) {
+#pragma unroll
+        for (int i = 0; i < NROW; ++i) {
+            l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
+            l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
+        }
+        if (KSPLIT > 1) {
+            constexpr int REGS = NROW * (D / 4 + 2);
+            if (ks > 0) {
+                float *dst = s_merge + (size_t)(g * (KSPLIT - 1) + ks - 1) * C::MERGE_FLOATS_PER_WARP + lane;
+                int c = 0;
+#pragma unroll
+                for (int i = 0; i < NROW; ++i) {
+                    dst[32 * c++] = m_run[i];
+                    dst[32 * c++] = l_run[i];
+#pragma unroll
+                    for (int nd = 0; nd < D / 8; ++nd) {
+                        dst[32 * c++] = oacc[nd][2 * i];
+                        dst[32 * c++] = oacc[nd][2 * i + 1];
+                    }
+                }
+                (void)REGS;
+            }
+            consumer_bar(NCW * 32);
+            if (ks == 0) {
+                for (int o = 0; o < KSPLIT - 1; ++o) {
+                    const float *src = s_merge + (size_t)(g * (KSPLIT - 1) + o) * C::MERGE_FLOATS_PER_WARP + lane;
+                    int c = 0;
+#pragma unroll
+                    for (int i = 0; i < NROW; ++i) {
+                        const float m2 = src[32 * c++];
+                        const float l2 = src[32 * c++];
+                        const float mn = fmaxf(m_run[i], m2);
+                        const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
+                        l_run[i] = l_run[i] * a + l2 * b;
+                        m_run[i] = mn;
+#pragma unroll
+                        for (int nd = 0; nd < D / 8; ++nd) {
+                            oacc[nd][2 * i] = oacc[nd][2 * i] * a + src[32 * c++] * b;
+                            oacc[nd][2 * i + 1] = oacc[nd][2 * i + 1] * a + src[32 * c++] * b;
+                        }
+                    }
+                }
+            }
+            consumer_bar(NCW * 32);
+        }
+        if (ks == 0) {
+            const bool whole = (ustart == s_P[r]) && (uend == s_P[r + 1]);
+#pragma unroll
+            for (int i = 0; i < NROW; ++i) {
+                const int hl = gid + 8 * i;
+                if (hl >= G) continue;
+                const int h = g * G + hl;
+                if (whole) {
+                    const float inv = l_run[i] > 0.f ? 1.0f / l_run[i] : 0.f;
+                    float *o = p.out + ((int64_t)r * p.Hq + h) * D;
+#pragma unroll
+                    for (int nd = 0; nd < D / 8; ++nd)
+                        *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) =
+                            make_float2(oacc[nd][2 * i] * inv, oacc[nd][2 * i + 1] * inv);
+                } else {
+                    const int slot = 2 * (int)blockIdx.x + ((s_P[r] <= u0) ? 0 : 1);
+                    float *base = p.partials + (size_t)slot * p.Hq * (D + 2);
+                    float *o = base + (size_t)h * D;
+#pragma unroll
+                    for (int nd = 0; nd < D / 8; ++nd)
+                        *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) = make_float2(oacc[nd][2 * i], oacc[nd][2 * i + 1]);
+                    if (t == 0) {
+                        base[(size_t)p.Hq * D + h] = m_run[i];
+                        base[(size_t)p.Hq * (D + 1) + h] = l_run[i];
+                    }
+                }
+            }
+        }
+    };
+
+    int r = find_region(s_P, n, u0);
+    int seg_start = u0;
+    int len = p.lens[r];
+    load_q(r);
+    int it = 0;
+    bool ok = true;
+    for (int u = u0; u < u1; ++u, ++it) {
+        if (u >= s_P[r + 1]) {
+            flush(r, seg_start, u);
+            while (u >= s_P[r + 1]) ++r;
+            seg_start = u;
+            len = p.lens[r];
+            load_q(r);
+        }
+        const int s = it % kStages;
+        ok = mbar_wait(smem_u32(&s_bar[s]), (it / kStages) & 1, &s_abort, p.status, 2);
+        if (!ok) break;
+        const int j0 = (u - s_P[r]) * CH + ks * 16;  // first row of this warp's block inside the region
+        if (j0 < len) {
+            const uint32_t k_base = smem_u32(s_stage + s * C::STAGE_BYTES) + g * C::HALVES * C::SUBTILE;
+            const uint32_t v_base = k_base + C::KV_BYTES;
+            const int mi = lane >> 3, rr = lane & 7;
+
+            // ---- S = Q K^T for 16 keys ----
+            float sacc[2][4];
+#pragma unroll
+            for (int a = 0; a < 2; ++a) sacc[a][0] = sacc[a][1] = sacc[a][2] = sacc[a][3] = 0.f;
+            {
+                const int row = ks * 16 + (mi >> 1) * 8 + rr;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const int hf = kk >> 2, chunk = ((kk & 3) << 1) + (mi & 1);
+                    uint32_t b[4];
+                    ldmatrix_x4(b, k_base + hf * C::SUBTILE + row * 128 + ((chunk ^ (row & 7)) << 4));
+                    mma_bf16_16816(sacc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[0], b[1]);
+                    mma_bf16_16816(sacc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[2], b[3]);
+                }
+            }
+            // ---- online softmax (exp2 domain) ----
+            const bool tail = j0 + 16 > len;
+            uint32_t pa[4];
+            float corr[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                if (i >= NROW) { pa[i] = 0u; pa[i + 2] = 0u; corr[i] = 1.f; continue; }
+                float x[4];
+                x[0] = sacc[0][2 * i] * p.sl2; x[1] = sacc[0][2 * i + 1] * p.sl2;
+                x[2] = sacc[1][2 * i] * p.sl2; x[3] = sacc[1][2 * i + 1] * p.sl2;
+                if (tail) {
+                    const int jk = j0 + 2 * t;
+                    if (jk >= len) x[0] = -INFINITY;
+                    if (jk + 1 >= len) x[1] = -INFINITY;
+                    if (jk + 8 >= len) x[2] = -INFINITY;
+                    if (jk + 9 >= len) x[3] = -INFINITY;
+                }
+                float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float mn = fmaxf(m_run[i], mx);  // finite: row j0 of the block is valid
+                corr[i] = exp2_or_zero(m_run[i], mn);
+                m_run[i] = mn;
+                pa[i] = pack_bf16(fast_exp2(x[0] - mn), fast_exp2(x[1] - mn));
+                pa[i + 2] = pack_bf16(fast_exp2(x[2] - mn), fast_exp2(x[3] - mn));
+                // the row sum uses the bf16-rounded probabilities the PV product sees
+                l_run[i] = l_run[i] * corr[i] + ((bf16lo(pa[i]) + bf16hi(pa[i])) + (bf16lo(pa[i + 2]) + bf16hi(pa[i + 2])));
+            }
+            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                for (int nd = 0; nd < D / 8; ++nd) {
+                    oacc[nd][0] *= corr[0]; oacc[nd][1] *= corr[0];
+                    if (G_HI) { oacc[nd][2] *= corr[1]; oacc[nd][3] *= corr[1]; }
+                }
+            }
+            // ---- O += P V ----
+            uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
+            if (tail) {
+                // rows past the region's end may hold anything (slack is never written): clear them so that
+                // 0 * garbage cannot turn into NaN
+                const int jk = j0 + 2 * t;
+                vmask0 = (jk < len ? 0x0000ffffu : 0u) | (jk + 1 < len ? 0xffff0000u : 0u);
+                vmask1 = (jk + 8 < len ? 0x0000ffffu : 0u) | (jk + 9 < len ? 0xffff0000u : 0u);
+            }
+            {
+                const int row = ks * 16 + (mi & 1) * 8 + rr;
+#pragma unroll
+                for (int n2 = 0; n2 < D / 16; ++n2) {
+                    const int cg = n2 * 2 + (mi >> 1);
+                    const int hf = cg >> 3, chunk = cg & 7;
+                    uint32_t b[4];
+                    ldmatrix_x4_trans(b, v_base + hf * C::SUBTILE + row * 128 + ((chunk ^ (row & 7)) << 4));
+                    if (tail) { b[0] &= vmask0; b[1] &= vmask1; b[2] &= vmask0; b[3] &= vmask1; }
+                    mma_bf16_16816(oacc[2 * n2], pa[0], pa[1], pa[2], pa[3], b[0], b[1]);
+                    mma_bf16_16816(oacc[2 * n2 + 1], pa[0], pa[1], pa[2], pa[3], b[2], b[3]);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_bar[kStages + s]));
+    }
+    if (ok) flush(r, seg_start, u1);
+}
+
+// Merges the partials of every region that more than one CTA worked on.  grid = regions, 128 threads.
+template <int D>
+__global__ void __launch_bounds__(128) combine_kernel(DecodeParams p, int n_ctas) {
+    const int r = blockIdx.x;
+    const int n = p.n_regions;
+    const int P0 = p.plan[r], P1 = p.plan[r + 1], total = p.plan[n];
+    float *o = p.out + (int64_t)r * p.Hq * D;
+    if (P1 == P0) {
+        for (int i = threadIdx.x; i < p.Hq * D; i += blockDim.x) o[i] = 0.f;
+        return;
+    }
+    const int upc = max(1, (total + n_ctas - 1) / n_ctas);
+    const int c0 = P0 / upc, c1 = (P1 - 1) / upc;
+    if (c0 == c1) return;  // finished inside the decode kernel
+    const size_t slot_floats = (size_t)p.Hq * (D + 2);
+    for (int i = threadIdx.x; i < p.Hq * D; i += blockDim.x) {
+        const int h = i / D;
+        float m_tot = -INFINITY;
+        for (int c = c0; c <= c1; ++c) {
+            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
+            m_tot = fmaxf(m_tot, p.partials[slot * slot_floats + (size_t)p.Hq * D + h]);
+        }
+        float num = 0.f, den = 0.f;
+        for (int c = c0; c <= c1; ++c) {
+            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
+            const float *base = p.partials + slot * slot_floats;
+            const float w = exp2_or_zero(base[(size_t)p.Hq * D + h], m_tot);
+            num += base[i] * w;
+            den += base[(size_t)p.Hq * (D + 1) + h] * w;
+        }
+        o[i] = den > 0.f ? num / den : 0.f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    }();
+    return fn;
+}
+
+// bf16 [rows, Hkv, D] viewed as a 3-D tensor (D, Hkv, rows); one box = 64 channels x 1 head x ch rows.
+int make_map(CUtensorMap *tm, const void *base, int D, int Hkv, int64_t rows, int ch) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) { set_last_cuda_error(cudaErrorSymbolNotFound); return AIRCACHE_ERR_CUDA; }
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)ch};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) { set_last_cuda_error(cudaErrorInvalidValue); return AIRCACHE_ERR_CUDA; }
+    return AIRCACHE_OK;
+}
+
+int sm_count(int *out) {
+    int dev = 0;
+    AIRCACHE_CUDA_TRY(cudaGetDevice(&dev));
+    AIRCACHE_CUDA_TRY(cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, dev));
+    return AIRCACHE_OK;
+}
+
+template <int D, int HKV, bool G_HI>
+int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
+    using C = DecodeCfg<D, HKV, G_HI>;
+    CUtensorMap tm_k, tm_v;
+    int rc = make_map(&tm_k, c->k, D, HKV, c->total_rows, C::CH);
+    if (rc) return rc;
+    if ((rc = make_map(&tm_v, c->v, D, HKV, c->total_rows, C::CH))) return rc;
+    int sms = 0;
+    if ((rc = sm_count(&sms))) return rc;
+    const int ctas = sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas;
+    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, HKV, G_HI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           C::SMEM_BYTES));
+    decode_kernel<D, HKV, G_HI><<<ctas, C::THREADS, C::SMEM_BYTES, st>>>(tm_k, tm_v, p);
+    AIRCACHE_LAUNCH_CHECK();
+    combine_kernel<D><<<p.n_regions, 128, 0, st>>>(p, ctas);
+    AIRCACHE_LAUNCH_CHECK();
+    return AIRCACHE_OK;
+}
+
+template <int D, int HKV>
+int launch_decode_g(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
+    return p.G > 8 ? launch_decode_t<D, HKV, true>(c, p, st) : launch_decode_t<D, HKV, false>(c, p, st);
+}
+
+template <int D>
+int launch_decode_d(const aircache_shape_t *s, const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
+    switch (s->n_kv_heads) {
+        case 1: return launch_decode_g<D, 1>(c, p, st);
+        case 2: return launch_decode_g<D, 2>(c, p, st);
+        case 4: return launch_decode_g<D, 4>(c, p, st);
+        case 8: return launch_decode_g<D, 8>(c, p, st);
+        default: return AIRCACHE_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace
+
+int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out, void *ws,
+                  cudaStream_t st) {
+    const WsLayout w = ws_layout(s);
+    DecodeParams p;
+    p.q = (const uint16_t *)q;
+    p.out = out;
+    p.offsets = c->offsets;
+    p.lens = c->lens;
+    p.plan = ws_ptr<int32_t>(ws, w.plan);
+    p.partials = ws_ptr<float>(ws, w.partials);
+    p.status = ws_ptr<uint32_t>(ws, w.status);
+    p.n_regions = s->n_layers * s->batch;
+    p.Hq = s->n_q_heads;
+    p.G = s->n_q_heads / s->n_kv_heads;
+    p.sl2 = s->scale * kLog2e;
+    return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
+}
+
+}  // namespace aircache

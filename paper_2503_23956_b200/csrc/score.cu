@@ -1,0 +1,386 @@
+// aircache_score: importance of every visual token seen from the elite observation window
+// (Section 3.3, Eq. 4-8), all layers and sequences per launch.
+//
+// Three kernels on one stream:
+//   elite_kernel       one CTA per (layer, sequence, KV head): Eq. 4 logits of the last text query against
+//                      the W candidate keys (fp64 dot products, so the Eq. 5 decision does not depend on a
+//                      summation order), the elite set of each query head, the list of elite rows
+//                      (head, window slot) of the KV group, and each row's softmax statistics over the
+//                      text keys it may see (elite, causal).
+//   stats_kernel       Eq. 7 pass one: Q_tk K_v^T on tensor cores (keys on the M axis, elite rows on N),
+//                      running (max, sum of exp2) of every elite row over one chunk of visual keys.
+//   importance_kernel  Eq. 7 pass two + Eq. 8: recomputes the same tiles (keys now come from L2), turns
+//                      logits into probabilities with the merged statistics and sums the rows of all heads
+//                      per key with weight 1 / (|E_h| Hq).  KV heads are visited in ascending order by one
+//                      thread per key, so the sum has a fixed order.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace aircache {
+
+namespace {
+
+struct ScoreParams {
+    const uint16_t *k;
+    int64_t s_layer, s_batch, s_head, s_token;
+    const uint16_t *qw;  // [L,B,W,Hq,d]
+    float *scores;       // [L,B,Nv]
+    uint64_t *elite_mask;
+    int32_t *row_count;
+    int32_t *row_info;
+    float *row_coef;
+    float2 *row_text;
+    float2 *chunk_stats;
+    int L, B, Hq, Hkv, G, d, Nv, Nt, W;
+    int cap, chunks, chunk_keys;
+    float scale, sl2, ln_alpha;
+    int keep_all;
+};
+
+constexpr float kNegBig = -1.0e30f;
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 4-5 and the elite-row table
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
+    __shared__ float s_logit[kMaxGroup * kMaxWindow];
+    __shared__ uint64_t s_mask[kMaxGroup];
+    __shared__ int s_first_row[kMaxGroup + 1];
+
+    const int grp = blockIdx.x;  // (l*B + b)*Hkv + g
+    const int g = grp % p.Hkv;
+    const int lb = grp / p.Hkv;
+    const int l = lb / p.B, b = lb % p.B;
+    const int N = p.Nv + p.Nt;
+    const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
+    const uint16_t *k_cand = k_g + (int64_t)(N - p.W) * p.s_token;
+    const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * p.d;
+
+    // Eq. 4, last row only: logit of candidate w for head hl, fp64 dot product in element order.
+    for (int idx = threadIdx.x; idx < p.G * p.W; idx += blockDim.x) {
+        const int hl = idx / p.W, w = idx % p.W;
+        const uint16_t *q = q_lb + ((int64_t)(p.W - 1) * p.Hq + g * p.G + hl) * p.d;
+        const uint16_t *kk = k_cand + (int64_t)w * p.s_token;
+        double acc = 0.0;
+        for (int c = 0; c < p.d; ++c) acc = __dadd_rn(acc, __dmul_rn((double)bf16_to_f32(q[c]), (double)bf16_to_f32(kk[c])));
+        s_logit[idx] = __fmul_rn((float)acc, p.scale);
+    }
+    __syncthreads();
+
+    // Eq. 5: candidates within a factor alpha of the best one (compared in the log domain, fp32).
+    if (threadIdx.x < p.G) {
+        const int hl = threadIdx.x;
+        const float *t = s_logit + hl * p.W;
+        float tmax = -INFINITY;
+        for (int w = 0; w < p.W; ++w) tmax = fmaxf(tmax, t[w]);
+        uint64_t mask = 0;
+        for (int w = 0; w < p.W; ++w) {
+            const float diff = __fsub_rn(t[w], tmax);
+            if (p.keep_all || diff >= p.ln_alpha) mask |= (uint64_t)1 << w;
+        }
+        s_mask[hl] = mask;
+        if (p.elite_mask) p.elite_mask[(int64_t)lb * p.Hq + g * p.G + hl] = mask;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int r = 0;
+        for (int hl = 0; hl < p.G; ++hl) {
+            s_first_row[hl] = r;
+            r += __popcll(s_mask[hl]);
+        }
+        s_first_row[p.G] = r;
+        p.row_count[grp] = r;
+    }
+    __syncthreads();
+
+    // Row table: elite rows of head hl are consecutive, ascending window slot.
+    int32_t *info = p.row_info + (int64_t)grp * p.cap;
+    float *coef = p.row_coef + (int64_t)grp * p.cap;
+    float2 *text = p.row_text + (int64_t)grp * p.cap;
+    for (int idx = threadIdx.x; idx < p.G * p.W; idx += blockDim.x) {
+        const int hl = idx / p.W, w = idx % p.W;
+        const uint64_t mask = s_mask[hl];
+        if (!((mask >> w) & 1)) continue;
+        const int r = s_first_row[hl] + __popcll(mask & (((uint64_t)1 << w) - 1));
+        info[r] = (hl << 8) | w;
+        coef[r] = 1.0f / ((float)__popcll(mask) * (float)p.Hq);
+        // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.
+        const uint16_t *q = q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * p.d;
+        float m = kNegBig, z = 0.0f;
+        for (int w2 = 0; w2 <= w; ++w2) {
+            if (!((mask >> w2) & 1)) continue;
+            const uint16_t *kk = k_cand + (int64_t)w2 * p.s_token;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            for (int c = 0; c < p.d; c += 4) {
+                a0 = fmaf(bf16_to_f32(q[c]), bf16_to_f32(kk[c]), a0);
+                a1 = fmaf(bf16_to_f32(q[c + 1]), bf16_to_f32(kk[c + 1]), a1);
+                a2 = fmaf(bf16_to_f32(q[c + 2]), bf16_to_f32(kk[c + 2]), a2);
+                a3 = fmaf(bf16_to_f32(q[c + 3]), bf16_to_f32(kk[c + 3]), a3);
+            }
+            merge_stats(m, z, ((a0 + a1) + (a2 + a3)) * p.sl2, 1.0f);
+        }
+        text[r] = make_float2(m, z);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-core tile shared by both passes.
+//
+// One warp computes S^T = K_tile (16 keys x d) * Q^T (d x 8*NT elite rows) with mma.m16n8k16.  The
+// contraction index is permuted inside each block of 32 channels so that every thread feeds the MMA
+// from one 16-byte load: thread t of a quad owns channels 8t..8t+7 of the block, both for the key rows
+// (read straight from global memory) and for the query rows (shared memory).  A dot product does not
+// depend on the order of its terms' indices as long as both operands use the same order.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+struct KeyFrag {
+    uint4 lo[D / 32];  // key row gid
+    uint4 hi[D / 32];  // key row gid + 8
+};
+
+template <int D>
+__device__ __forceinline__ void load_keys(KeyFrag<D> &f, const uint16_t *row_lo, const uint16_t *row_hi, int t) {
+#pragma unroll
+    for (int kb = 0; kb < D / 32; ++kb) {
+        f.lo[kb] = __ldg(reinterpret_cast<const uint4 *>(row_lo + kb * 32 + 8 * t));
+        f.hi[kb] = __ldg(reinterpret_cast<const uint4 *>(row_hi + kb * 32 + 8 * t));
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void tile_mma(float (&acc)[4], const KeyFrag<D> &f, const uint16_t *q_row, int t) {
+    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll
+    for (int kb = 0; kb < D / 32; ++kb) {
+        const uint4 bq = *reinterpret_cast<const uint4 *>(q_row + kb * 32 + 8 * t);
+        mma_bf16_16816(acc, f.lo[kb].x, f.hi[kb].x, f.lo[kb].y, f.hi[kb].y, bq.x, bq.y);
+        mma_bf16_16816(acc, f.lo[kb].z, f.hi[kb].z, f.lo[kb].w, f.hi[kb].w, bq.z, bq.w);
+    }
+}
+
+// Copies up to 8*NT elite query rows (starting at row0) of one KV group into shared memory, zero padded.
+template <int D>
+__device__ __forceinline__ void stage_queries(uint16_t *s_q, const ScoreParams &p, int grp, int lb, int g,
+                                              int row0, int n_rows_total, int rows_pad) {
+    constexpr int QS = D + 32;
+    const int32_t *info = p.row_info + (int64_t)grp * p.cap;
+    const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * D;
+    for (int idx = threadIdx.x; idx < rows_pad * (D / 8); idx += blockDim.x) {
+        const int r = idx / (D / 8), c = idx % (D / 8);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row0 + r < n_rows_total) {
+            const int in = info[row0 + r];
+            const int hl = in >> 8, w = in & 255;
+            v = __ldg(reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D) + c);
+        }
+        *reinterpret_cast<uint4 *>(s_q + r * QS + c * 8) = v;
+    }
+}
+
+// Eq. 7, pass one.  grid = (chunks, L*B*Hkv), 128 threads.
+template <int D, int NT>
+__global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
+    constexpr int QS = D + 32;
+    __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
+    __shared__ float2 s_red[4][NT * 8];
+
+    const int grp = blockIdx.y;
+    const int g = grp % p.Hkv;
+    const int lb = grp / p.Hkv;
+    const int l = lb / p.B, b = lb % p.B;
+    const int chunk = blockIdx.x;
+    const int key0 = chunk * p.chunk_keys;
+    const int key1 = min(p.Nv, key0 + p.chunk_keys);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
+    const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
+    const int n_rows = p.row_count[grp];
+    float2 *out = p.chunk_stats + ((int64_t)grp * p.chunks + chunk) * p.cap;
+
+    for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
+        const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
+        __syncthreads();
+        stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
+        __syncthreads();
+
+        float m[NT][2], z[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = kNegBig; z[nt][0] = z[nt][1] = 0.f; }
+
+        for (int kt = key0 + warp * 16; kt < key1; kt += 64) {
+            const int ka = kt + gid, kb = kt + gid + 8;
+            const bool va = ka < key1, vb = kb < key1;
+            KeyFrag<D> f;
+            load_keys<D>(f, k_g + (int64_t)(va ? ka : key1 - 1) * p.s_token,
+                         k_g + (int64_t)(vb ? kb : key1 - 1) * p.s_token, t);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (nt < nt_used) {
+                    float acc[4];
+                    tile_mma<D>(acc, f, s_q + (nt * 8 + gid) * QS, t);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const float xa = va ? acc[j] * p.sl2 : kNegBig;
+                        const float xb = vb ? acc[j + 2] * p.sl2 : kNegBig;
+                        const float mn = fmaxf(m[nt][j], fmaxf(xa, xb));
+                        const float ea = va ? fast_exp2(xa - mn) : 0.f;
+                        const float eb = vb ? fast_exp2(xb - mn) : 0.f;
+                        z[nt][j] = z[nt][j] * fast_exp2(m[nt][j] - mn) + (ea + eb);
+                        m[nt][j] = mn;
+                    }
+                }
+            }
+        }
+        // combine the eight key lanes of a column, then the four warps, in a fixed order
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            if (nt < nt_used) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    float mm = m[nt][j], zz = z[nt][j];
+#pragma unroll
+                    for (int sh = 4; sh < 32; sh <<= 1) {
+                        const float m2 = __shfl_xor_sync(0xffffffffu, mm, sh);
+                        const float z2 = __shfl_xor_sync(0xffffffffu, zz, sh);
+                        merge_stats(mm, zz, m2, z2);
+                    }
+                    if (gid == 0) s_red[warp][nt * 8 + 2 * t + j] = make_float2(mm, zz);
+                }
+            }
+        }
+        __syncthreads();
+        for (int r = threadIdx.x; r < nt_used * 8; r += blockDim.x) {
+            float2 a = s_red[0][r];
+#pragma unroll
+            for (int w2 = 1; w2 < 4; ++w2) merge_stats(a.x, a.y, s_red[w2][r].x, s_red[w2][r].y);
+            if (row0 + r < n_rows) out[row0 + r] = a;
+        }
+    }
+}
+
+// Eq. 7 pass two and Eq. 8.  grid = (ceil(Nv / 128), L*B), 128 threads; each warp owns 32 keys.
+template <int D, int NT>
+__global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
+    constexpr int QS = D + 32;
+    __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
+    __shared__ float2 s_stat[NT * 8];  // (row max, weight / normaliser)
+
+    const int lb = blockIdx.y;
+    const int l = lb / p.B, b = lb % p.B;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
+    const int kbase = blockIdx.x * kScoreKeyTile + warp * 32;
+    float imp[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [m-tile][key gid / gid+8]
+
+    for (int g = 0; g < p.Hkv; ++g) {
+        const int grp = lb * p.Hkv + g;
+        const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
+        const int n_rows = p.row_count[grp];
+        KeyFrag<D> f[2];
+        bool valid[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int ka = kbase + mt * 16 + gid, kb = ka + 8;
+            valid[mt][0] = ka < p.Nv;
+            valid[mt][1] = kb < p.Nv;
+            load_keys<D>(f[mt], k_g + (int64_t)(valid[mt][0] ? ka : p.Nv - 1) * p.s_token,
+                         k_g + (int64_t)(valid[mt][1] ? kb : p.Nv - 1) * p.s_token, t);
+        }
+        for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
+            const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
+            __syncthreads();
+            stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
+            for (int r = threadIdx.x; r < nt_used * 8; r += blockDim.x) {
+                float2 st = make_float2(0.f, 0.f);
+                if (row0 + r < n_rows) {
+                    const float2 tx = p.row_text[(int64_t)grp * p.cap + row0 + r];
+                    float m = tx.x, z = tx.y;
+                    for (int c = 0; c < p.chunks; ++c) {
+                        const float2 cs = p.chunk_stats[((int64_t)grp * p.chunks + c) * p.cap + row0 + r];
+                        merge_stats(m, z, cs.x, cs.y);
+                    }
+                    st = make_float2(m, p.row_coef[(int64_t)grp * p.cap + row0 + r] / z);
+                }
+                s_stat[r] = st;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (nt < nt_used) {
+                    const float2 s0 = s_stat[nt * 8 + 2 * t], s1 = s_stat[nt * 8 + 2 * t + 1];
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        float acc[4];
+                        tile_mma<D>(acc, f[mt], s_q + (nt * 8 + gid) * QS, t);
+                        imp[mt][0] += fast_exp2(acc[0] * p.sl2 - s0.x) * s0.y + fast_exp2(acc[1] * p.sl2 - s1.x) * s1.y;
+                        imp[mt][1] += fast_exp2(acc[2] * p.sl2 - s0.x) * s0.y + fast_exp2(acc[3] * p.sl2 - s1.x) * s1.y;
+                    }
+                }
+            }
+        }
+    }
+    float *out = p.scores + (int64_t)lb * p.Nv;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float v = imp[mt][j];
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            v += __shfl_xor_sync(0xffffffffu, v, 2);
+            const int key = kbase + mt * 16 + gid + 8 * j;
+            if (t == 0 && key < p.Nv) out[key] = v;
+        }
+    }
+}
+
+template <int D, int NT>
+int launch_passes(const ScoreParams &p, cudaStream_t st) {
+    const int64_t LB = (int64_t)p.L * p.B;
+    stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)(LB * p.Hkv)), 128, 0, st>>>(p);
+    AIRCACHE_LAUNCH_CHECK();
+    importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)LB), 128, 0, st>>>(p);
+    AIRCACHE_LAUNCH_CHECK();
+    return AIRCACHE_OK;
+}
+
+template <int D>
+int launch_passes_d(const ScoreParams &p, cudaStream_t st) {
+    const int nt_max = (p.G * p.W + 7) / 8;
+    if (nt_max <= 2) return launch_passes<D, 2>(p, st);
+    if (nt_max <= 4) return launch_passes<D, 4>(p, st);
+    if (nt_max <= 8) return launch_passes<D, 8>(p, st);
+    return launch_passes<D, 16>(p, st);
+}
+
+}  // namespace
+
+int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void *q_window, float alpha,
+                 float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st) {
+    const WsLayout w = ws_layout(s);
+    ScoreParams p;
+    p.k = (const uint16_t *)f->k;
+    p.s_layer = f->stride_layer; p.s_batch = f->stride_batch; p.s_head = f->stride_head; p.s_token = f->stride_token;
+    p.qw = (const uint16_t *)q_window;
+    p.scores = scores;
+    p.elite_mask = elite_mask;
+    p.row_count = ws_ptr<int32_t>(ws, w.row_count);
+    p.row_info = ws_ptr<int32_t>(ws, w.row_info);
+    p.row_coef = ws_ptr<float>(ws, w.row_coef);
+    p.row_text = ws_ptr<float2>(ws, w.row_text);
+    p.chunk_stats = ws_ptr<float2>(ws, w.chunk_stats);
+    p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
+    p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
+    p.cap = score_row_cap(s);
+    p.chunks = score_chunks(s);
+    p.chunk_keys = (int)align_up((s->n_visual + p.chunks - 1) / p.chunks, 16);
+    p.scale = s->scale;
+    p.sl2 = s->scale * kLog2e;
+    p.keep_all = alpha <= 0.0f;
+    p.ln_alpha = p.keep_all ? 0.0f : (float)log((double)alpha);
+
+    const int64_t groups = (int64_t)p.L * p.B * p.Hkv;
+    elite_kernel<<<(unsigned)groups, 128, 0, st>>>(p);
+    AIRCACHE_LAUNCH_CHECK();
+    return s->head_dim == 64 ? launch_passes_d<64>(p, st) : launch_passes_d<128>(p, st);
+}
+
+}  // namespace aircache

@@ -1,0 +1,416 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on the same seeded
+inputs.  Integer results (elite masks, budgets, offsets, kept-token lists, gathered bytes) must be equal;
+floating-point results must agree within 2e-3 (scores: element-wise relative; attention outputs: per row,
+max |a - b| / max |b|).  Stage-isolated tests feed a CUDA stage the oracle's upstream output, so the
+integer stages are compared on identical input bits; end-to-end tests chain the CUDA stages."""
+import numpy as np
+import pytest
+import torch
+
+from workloads import CONFIGS, Workload, decode_queries
+
+from harness import GpuPath, gen_inputs, logical, oracle_dims, rel_elem_err, rel_row_err, u16
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+DEV = "cuda:0"
+
+
+def small(name, L=3, Hq=28, Hkv=4, d=128, B=2, Nv=1000, Nt=40, ratio=0.1, W=16, **kw):
+    return Workload(name, L, Hq, Hkv, d, batch=B, n_visual=Nv, n_text=Nt, ratio=ratio, steps=2, window=W, **kw)
+
+
+CASES = {
+    "c1": CONFIGS["c1"],
+    "s7b": small("s7b"),                                           # 7B head layout, ragged tails everywhere
+    "s72b": small("s72b", L=2, Hq=64, Hkv=8, B=2, Nv=777, Nt=33),   # 72B head layout
+    "mha64": small("mha64", L=2, Hq=4, Hkv=4, d=64, B=3, Nv=300, Nt=20, W=8),
+    "g16": small("g16", L=2, Hq=16, Hkv=1, d=64, B=2, Nv=257, Nt=17, W=5),   # 16 query heads per KV head
+    "kv2": small("kv2", L=2, Hq=12, Hkv=2, d=128, B=2, Nv=515, Nt=64, W=64),  # widest window
+    "kv1": small("kv1", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=130, Nt=9, W=9),
+}
+
+
+@pytest.fixture(scope="module")
+def oracle(oracle_mod):
+    return oracle_mod
+
+
+def cpu_inputs(wl):
+    return gen_inputs(wl, "cpu")
+
+
+_ORACLE_CACHE = {}
+
+
+def oracle_path(oracle, wl, ratio=None, alpha=None, slack=0, mode=0):
+    """Chained oracle: scores -> moments -> budgets -> compact.  Cached per argument tuple."""
+    key = (wl, ratio, alpha, slack, mode)
+    if key in _ORACLE_CACHE:
+        return _ORACLE_CACHE[key]
+    ratio = wl.ratio if ratio is None else ratio
+    alpha = wl.alpha if alpha is None else alpha
+    k, v, qw = cpu_inputs(wl)
+    dm = oracle_dims(oracle, wl)
+    kl, vl = u16(logical(k)), u16(logical(v))
+    sc = oracle.score(dm, kl, u16(qw), wl.scale, alpha)
+    st, sk = oracle.moments(sc["scores"])
+    bud = oracle.allocate(st, sk, wl.n_visual, ratio, mode)
+    cp = oracle.compact(dm, slack, kl, vl, sc["scores"], bud)
+    res = dict(k=k, v=v, qw=qw, dims=dm, scores=sc["scores"], mask=sc["elite_mask"], strength=st, skew=sk,
+               budgets=bud, compact=cp, ratio=ratio, alpha=alpha)
+    _ORACLE_CACHE[key] = res
+    return res
+
+
+def make_gpu(wl, ref, slack=0):
+    gp = GpuPath(wl, ratio=ref["ratio"], device=DEV, slack=slack)
+    gp.set_full(logical(ref["k"].to(DEV)), logical(ref["v"].to(DEV)))
+    return gp
+
+
+def compare_cache(gp, cp):
+    """Valid rows of K'/V', offsets, lens and kept lists are bit-identical to the oracle's."""
+    assert np.array_equal(gp.offsets.cpu().numpy(), cp["offsets"])
+    assert np.array_equal(gp.lens.cpu().numpy(), cp["lens"])
+    kc, vc = u16(gp.k_c), u16(gp.v_c)
+    for r in range(len(cp["lens"])):
+        a, n = int(cp["offsets"][r]), int(cp["lens"][r])
+        assert np.array_equal(kc[a:a + n], cp["k"][a:a + n]), f"K' region {r}"
+        assert np.array_equal(vc[a:a + n], cp["v"][a:a + n]), f"V' region {r}"
+
+
+# --------------------------------------------------------------------------------------------------
+# stage-isolated parity
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("alpha", [0.9, 0.0, 1.0])
+def test_score_parity(oracle, case, alpha):
+    wl = CASES[case]
+    if alpha != 0.9 and case in ("s72b",):
+        pytest.skip("alpha sweep covered by the smaller cases")
+    ref = oracle_path(oracle, wl, alpha=alpha)
+    gp = make_gpu(wl, ref)
+    gp.score(ref["qw"].to(DEV), alpha=alpha)
+    assert gp.status() == 0
+    mask = gp.mask.cpu().numpy().view(np.uint64)
+    assert np.array_equal(mask, ref["mask"]), "elite sets differ"
+    err = rel_elem_err(gp.scores.cpu().numpy(), ref["scores"])
+    assert err <= TOL, err
+
+
+@pytest.mark.parametrize("case", ["c1", "s7b", "mha64"])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("ratio", [0.1, 0.83])
+def test_budget_parity_on_oracle_scores(oracle, case, mode, ratio):
+    wl = CASES[case]
+    ref = oracle_path(oracle, wl, ratio=ratio, mode=mode, slack=3)
+    gp = make_gpu(wl, ref, slack=3)
+    gp.budget(scores=torch.from_numpy(ref["scores"]).to(DEV), mode=mode)
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+    assert np.allclose(gp.strength.cpu().numpy(), ref["strength"], rtol=1e-12, atol=0)
+    assert np.allclose(gp.skew.cpu().numpy(), ref["skew"], rtol=1e-9, atol=1e-12)
+    assert np.array_equal(gp.offsets.cpu().numpy(), ref["compact"]["offsets"])
+    assert np.array_equal(gp.lens.cpu().numpy(), ref["compact"]["lens"])
+    assert int(gp.budgets.sum()) == wl.batch * oracle.total_kept(wl.n_visual, wl.n_layers, ratio)
+
+
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("slack", [0, 5])
+def test_compact_parity_on_oracle_scores_and_budgets(oracle, case, slack):
+    wl = CASES[case]
+    ref = oracle_path(oracle, wl, slack=slack)
+    gp = make_gpu(wl, ref, slack=slack)
+    gp.budget(scores=torch.from_numpy(ref["scores"]).to(DEV))   # layout (offsets, lens) comes from the budget call
+    gp.compact(scores=torch.from_numpy(ref["scores"]).to(DEV), budgets=torch.from_numpy(ref["budgets"]).to(DEV))
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(ref["compact"]["kept_idx"])], ref["compact"]["kept_idx"])
+    compare_cache(gp, ref["compact"])
+
+
+def test_select_ties_zero_and_full_budgets(oracle):
+    """Heavily duplicated scores (ties broken by the lower index), a layer that keeps nothing and one that
+    keeps everything, negative zero and denormal scores; head-major source layout."""
+    wl = small("ties", L=4, Hq=8, Hkv=2, d=64, B=2, Nv=611, Nt=12, W=4)
+    rng = np.random.default_rng(7)
+    k, v, _ = cpu_inputs(wl)
+    scores = (rng.integers(0, 6, size=(wl.n_layers, wl.batch, wl.n_visual)) / 8.0).astype(np.float32)
+    scores[1, 0, :5] = [-0.0, 0.0, 1e-42, 1e-42, -0.0]
+    # a layer that keeps nothing, one that keeps one token, two that keep everything; both sequences sum to T
+    budgets = np.array([[0, 200], [300, wl.n_visual], [1, 100], [wl.n_visual, 1]], np.int32)
+    T = int(budgets[:, 0].sum())
+    assert T == int(budgets[:, 1].sum())
+    ratio = T / (wl.n_visual * wl.n_layers)
+    dm = oracle_dims(oracle, wl)
+    assert oracle.total_kept(wl.n_visual, wl.n_layers, ratio) == T
+    k_hm = k.permute(0, 1, 3, 2, 4).contiguous()    # head-major storage [L,B,Hkv,N,d]
+    v_hm = v.permute(0, 1, 3, 2, 4).contiguous()
+    cp = oracle.compact(dm, 2, u16(k_hm), u16(v_hm), scores, budgets)
+    gp = GpuPath(wl, ratio=ratio, device=DEV, slack=2)
+    gp.set_full(k_hm.to(DEV), v_hm.to(DEV))
+    sc_d, bud_d = torch.from_numpy(scores).to(DEV), torch.from_numpy(budgets).to(DEV)
+    # offsets/lens for these hand-made budgets: written here the way aircache_budget lays regions out
+    sizes = budgets.reshape(-1).astype(np.int64) + wl.n_text + 2
+    gp.offsets.copy_(torch.from_numpy(np.concatenate([[0], np.cumsum(sizes)])))
+    gp.lens.copy_(torch.from_numpy((budgets.reshape(-1) + wl.n_text).astype(np.int32)))
+    gp.compact(scores=sc_d, budgets=bud_d)
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+    # the same through the workspace-held index list
+    gp.k_c.zero_(); gp.v_c.zero_()
+    gp.compact(scores=sc_d, budgets=bud_d, want_kept=False)
+    compare_cache(gp, cp)
+
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_decode_parity_on_oracle_cache(oracle, case):
+    wl = CASES[case]
+    slack = 4
+    ref = oracle_path(oracle, wl, slack=slack)
+    cp = ref["compact"]
+    gp = make_gpu(wl, ref, slack=slack)
+    # poison everything, then upload only the valid rows: slack rows stay NaN and must not leak
+    gp.k_c.fill_(float("nan")); gp.v_c.fill_(float("nan"))
+    kc = torch.from_numpy(cp["k"].view(np.int16)).view(torch.bfloat16)
+    vc = torch.from_numpy(cp["v"].view(np.int16)).view(torch.bfloat16)
+    for r in range(len(cp["lens"])):
+        a, n = int(cp["offsets"][r]), int(cp["lens"][r])
+        gp.k_c[a:a + n] = kc[a:a + n].to(DEV)
+        gp.v_c[a:a + n] = vc[a:a + n].to(DEV)
+    gp.offsets.copy_(torch.from_numpy(cp["offsets"]))
+    gp.lens.copy_(torch.from_numpy(cp["lens"]))
+    for step in range(2):
+        q = decode_queries(wl, step, "cpu")
+        want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q), wl.scale)
+        gp.out.fill_(float("nan"))
+        gp.decode(q.to(DEV))
+        assert gp.status() == 0
+        got = gp.out.cpu().numpy()
+        assert np.isfinite(got).all()
+        err = rel_row_err(got, want)
+        assert err <= TOL, err
+
+
+def test_decode_tiny_and_empty_regions(oracle):
+    """Regions of 0, 1, 15, 16, 17 and 33 rows next to long ones."""
+    wl = small("tiny", L=2, Hq=28, Hkv=4, d=128, B=4, Nv=400, Nt=8, W=4)
+    rng = np.random.default_rng(11)
+    lens = np.array([0, 1, 15, 16, 17, 33, 300, 64], np.int32)
+    sizes = lens.astype(np.int64) + 3
+    offsets = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    rows = int(offsets[-1])
+    from workloads.synth import to_u16
+    kc = torch.from_numpy(rng.standard_normal((rows, 4, 128)).astype(np.float32)).to(torch.bfloat16)
+    vc = torch.from_numpy(rng.standard_normal((rows, 4, 128)).astype(np.float32)).to(torch.bfloat16)
+    q = decode_queries(wl, 0, "cpu")
+    dm = oracle_dims(oracle, wl)
+    want = oracle.decode(dm, to_u16(kc), to_u16(vc), offsets, lens, u16(q), wl.scale)
+    gp = GpuPath(wl, ratio=1.0, device=DEV, slack=3)
+    gp.k_c.fill_(float("nan")); gp.v_c.fill_(float("nan"))
+    for r in range(len(lens)):
+        a, n = int(offsets[r]), int(lens[r])
+        gp.k_c[a:a + n] = kc[a:a + n].to(DEV)
+        gp.v_c[a:a + n] = vc[a:a + n].to(DEV)
+    gp.offsets.copy_(torch.from_numpy(offsets)); gp.lens.copy_(torch.from_numpy(lens))
+    gp.out.fill_(float("nan"))
+    gp.decode(q.to(DEV))
+    assert gp.status() == 0
+    got = gp.out.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert (got.reshape(8, -1)[0] == 0).all()            # empty region -> zeros
+    assert rel_row_err(got, want) <= TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# end to end: CUDA stages chained, against the chained oracle
+# --------------------------------------------------------------------------------------------------
+def run_chain(gp, ref):
+    gp.score(ref["qw"].to(DEV), alpha=ref["alpha"])
+    gp.budget()
+    gp.compact()
+
+
+@pytest.mark.parametrize("case", ["c1", "s7b", "s72b", "kv2"])
+def test_end_to_end_chain(oracle, case):
+    wl = CASES[case]
+    ref = oracle_path(oracle, wl)
+    gp = make_gpu(wl, ref)
+    run_chain(gp, ref)
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"])
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+    cp = ref["compact"]
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+    q = decode_queries(wl, 0, "cpu")
+    want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q), wl.scale)
+    gp.decode(q.to(DEV))
+    assert gp.status() == 0
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+    # text rows are never evicted and sit after the kept visual rows, in order
+    kc = u16(gp.k_c)
+    kl = u16(logical(ref["k"]))
+    for r in range(len(cp["lens"])):
+        l, b = divmod(r, wl.batch)
+        a, n = int(cp["offsets"][r]), int(cp["lens"][r])
+        text = kl[l, b, :, wl.n_visual:, :].transpose(1, 0, 2)
+        assert np.array_equal(kc[a + n - wl.n_text:a + n], text)
+
+
+def test_full_retention_equals_full_cache_decode(oracle):
+    wl = CASES["s7b"]
+    ref = oracle_path(oracle, wl, ratio=1.0)
+    gp = make_gpu(wl, ref)
+    run_chain(gp, ref)
+    assert (gp.budgets.cpu().numpy() == wl.n_visual).all()
+    q = decode_queries(wl, 0, "cpu")
+    # full-cache reference: one region per (l, b) holding every token, straight from the generator output
+    L, B, N = wl.n_layers, wl.batch, wl.n_tokens
+    kf = u16(ref["k"]).reshape(L * B * N, wl.n_kv_heads, wl.head_dim)
+    vf = u16(ref["v"]).reshape(L * B * N, wl.n_kv_heads, wl.head_dim)
+    offs = (np.arange(L * B + 1) * N).astype(np.int64)
+    lens = np.full(L * B, N, np.int32)
+    want = oracle.decode(ref["dims"], kf, vf, offs, lens, u16(q), wl.scale)
+    gp.decode(q.to(DEV))
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+
+
+def test_results_are_bit_reproducible(oracle):
+    wl = CASES["s7b"]
+    ref = oracle_path(oracle, wl)
+    outs = []
+    for _ in range(2):
+        gp = make_gpu(wl, ref)
+        run_chain(gp, ref)
+        q = decode_queries(wl, 1, DEV)
+        gp.decode(q)
+        outs.append((gp.scores.cpu().numpy().copy(), gp.budgets.cpu().numpy().copy(),
+                     gp.kept.cpu().numpy().copy(), gp.out.cpu().numpy().copy()))
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+def test_append_then_decode(oracle):
+    """Eq. 2: three appended tokens per region land in the slack rows and take part in the next step."""
+    wl = CASES["s7b"]
+    slack = 3
+    ref = oracle_path(oracle, wl, slack=slack)
+    cp = ref["compact"]
+    gp = make_gpu(wl, ref, slack=slack)
+    run_chain(gp, ref)
+    import paper_2503_23956_b200 as ac
+    rng = np.random.default_rng(5)
+    k_o, v_o, lens = cp["k"].copy(), cp["v"].copy(), cp["lens"].copy()
+    LB = wl.n_layers * wl.batch
+    for i in range(slack):
+        kn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        vn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        ac.aircache_append(gp.sh, gp.cache, kn.to(DEV), vn.to(DEV), i)
+        for r in range(LB):
+            k_o[cp["offsets"][r] + lens[r]] = u16(kn)[r]
+            v_o[cp["offsets"][r] + lens[r]] = u16(vn)[r]
+        lens += 1
+    assert ac.aircache_append(gp.sh, gp.cache, kn.to(DEV), vn.to(DEV), slack, check=False) == ac.ERR_CAPACITY
+    assert np.array_equal(gp.lens.cpu().numpy(), lens)
+    q = decode_queries(wl, 0, "cpu")
+    want = oracle.decode(ref["dims"], k_o, v_o, cp["offsets"], lens, u16(q), wl.scale)
+    gp.decode(q.to(DEV))
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+
+
+def test_pipeline_host_matches_staged_calls(oracle):
+    import paper_2503_23956_b200 as ac
+    wl = CASES["c1"]
+    ref = oracle_path(oracle, wl)
+    gp = make_gpu(wl, ref)
+    run_chain(gp, ref)
+    n_steps = 3
+    q_steps = torch.stack([decode_queries(wl, s, "cpu") for s in range(n_steps)]).contiguous()
+    staged = []
+    for s in range(n_steps):
+        gp.decode(q_steps[s].to(DEV))
+        staged.append(gp.out.cpu().numpy().copy())
+    gp2 = GpuPath(wl, ratio=ref["ratio"], device=DEV)
+    h_k, h_v = ref["k"].contiguous().pin_memory(), ref["v"].contiguous().pin_memory()
+    h_full = ac.full_view(logical(h_k), logical(h_v))
+    d_k, d_v = torch.empty_like(h_k, device=DEV), torch.empty_like(h_v, device=DEV)
+    h_qw = ref["qw"].contiguous().pin_memory()
+    d_qw = torch.empty_like(h_qw, device=DEV)
+    h_q = q_steps.pin_memory()
+    d_q = torch.empty_like(h_q, device=DEV)
+    d_out = torch.empty((n_steps,) + tuple(gp.out.shape), dtype=torch.float32, device=DEV)
+    h_out = torch.empty(d_out.shape, dtype=torch.float32).pin_memory()
+    h_bud = torch.empty(gp.budgets.shape, dtype=torch.int32).pin_memory()
+    ac.aircache_pipeline_host(gp2.sh, h_full, h_k.numel(), d_k, d_v, h_qw, d_qw, h_q, d_q, n_steps, wl.alpha,
+                              ref["ratio"], 0, gp2.scores, gp2.budgets, gp2.cache, d_out, h_out, h_bud, gp2.ws)
+    assert np.array_equal(h_bud.numpy(), ref["budgets"])
+    for s in range(n_steps):
+        assert np.array_equal(h_out[s].numpy(), staged[s])
+
+
+# --------------------------------------------------------------------------------------------------
+# full-size configurations, in the launch configuration the benchmark times
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("ratio", [0.10, 0.50])
+def test_config2_full_size(oracle, ratio):
+    """Qwen2-7B-shaped single image (28 layers, 7290 + 128 tokens): the whole chain against the whole oracle."""
+    wl = CONFIGS["c2"]
+    ref = oracle_path(oracle, wl, ratio=ratio)
+    gp = make_gpu(wl, ref)
+    run_chain(gp, ref)
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"])
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+    cp = ref["compact"]
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+    for step in (0, 1):
+        q = decode_queries(wl, step, "cpu")
+        want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q), wl.scale)
+        gp.decode(q.to(DEV))
+        assert gp.status() == 0
+        assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+
+
+@pytest.mark.parametrize("cfg,batch,seqs", [("c3", 32, (0, 31)), ("c4", 4, (1,))])
+def test_batched_configs_sampled_sequences(oracle, cfg, batch, seqs):
+    """Batched 7B-shaped configurations at full batch on the GPU; the oracle runs whole sequences sampled
+    from the batch (every stage is independent per sequence, so a sequence's regions compare one to one)."""
+    from workloads import full_cache, window_queries
+    wl = CONFIGS[cfg].with_(batch=batch)
+    gp = GpuPath(wl, device=DEV)
+    k, v = full_cache(wl, "k", DEV), full_cache(wl, "v", DEV)
+    gp.set_full(logical(k), logical(v))
+    qw = window_queries(wl, DEV)
+    gp.score(qw)
+    gp.budget()
+    gp.compact()
+    q = decode_queries(wl, 0, DEV)
+    gp.decode(q)
+    assert gp.status() == 0
+    offs, lens = gp.offsets.cpu().numpy(), gp.lens.cpu().numpy()
+    kc, vc = u16(gp.k_c), u16(gp.v_c)
+    out = gp.out.cpu().numpy()
+    assert (gp.budgets.sum(dim=0).cpu().numpy() == oracle.total_kept(wl.n_visual, wl.n_layers, wl.ratio)).all()
+    for b in seqs:
+        w1 = wl.with_(batch=1)
+        dm = oracle_dims(oracle, w1)
+        kb, vb = full_cache(wl, "k", "cpu", seqs=[b]), full_cache(wl, "v", "cpu", seqs=[b])
+        qwb = window_queries(wl, "cpu", seqs=[b])
+        sc = oracle.score(dm, u16(logical(kb)), u16(qwb), wl.scale, wl.alpha)
+        assert np.array_equal(gp.mask[:, b].cpu().numpy().view(np.uint64), sc["elite_mask"][:, 0])
+        assert rel_elem_err(gp.scores[:, b].cpu().numpy(), sc["scores"][:, 0]) <= TOL
+        st, sk = oracle.moments(sc["scores"])
+        bud = oracle.allocate(st, sk, wl.n_visual, wl.ratio, 0)
+        assert np.array_equal(gp.budgets[:, b].cpu().numpy(), bud[:, 0])
+        cp = oracle.compact(dm, 0, u16(logical(kb)), u16(logical(vb)), sc["scores"], bud)
+        qb = decode_queries(wl, 0, "cpu", seqs=[b])
+        want = oracle.decode(dm, cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(qb), wl.scale)
+        for l in range(wl.n_layers):
+            r = l * wl.batch + b
+            a, n = int(offs[r]), int(lens[r])
+            a0, n0 = int(cp["offsets"][l]), int(cp["lens"][l])
+            assert n == n0
+            assert np.array_equal(kc[a:a + n], cp["k"][a0:a0 + n0])
+            assert np.array_equal(vc[a:a + n], cp["v"][a0:a0 + n0])
+        assert rel_row_err(out[:, b], want[:, 0]) <= TOL
