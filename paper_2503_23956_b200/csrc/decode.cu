@@ -15,7 +15,8 @@
 //   S = Q_g K^T   mma.m16n8k16: the G query heads of the group are the M rows (padded to 16), keys are N;
 //                 K fragments come from ldmatrix on the swizzled tile
 //   online softmax in the exp2 domain, warp-shuffle row maxima over the quad that shares a row
-//   O += P V      P rounded to bf16 (the row sum uses the same rounded values), V fragments from
+//   O += P V      P split into a bf16 head and a bf16 remainder (two MMAs per V fragment: a single bf16
+//                 rounding of P costs up to 2^-9 relative, too close to the 2e-3 bar), V fragments from
 //                 ldmatrix.trans
 // The G-fold reuse of every K/V row across the query heads of a group is what puts this on the tensor
 // pipe: with plain FMAs the kernel would need about 7 flop per byte, more than half of the fp32 peak at
@@ -109,7 +110,6 @@ __device__ __forceinline__ float exp2_or_zero(float m, float m_new) {
 template <int D, int HKV, bool G_HI>
 struct DecodeCfg {
     static constexpr int NROW = G_HI ? 2 : 1;        // accumulator row groups in use (heads 0-7, heads 8-15)
-    static constexpr int NSTAGE = G_HI ? 2 : 3;      // ring depth (the wider merge buffer costs one stage)
     static constexpr int KSPLIT = (8 / HKV) > 4 ? 4 : (8 / HKV);
     static constexpr int CH = 16 * KSPLIT;           // rows per unit
     static constexpr int NCW = HKV * KSPLIT;         // consumer warps
@@ -122,6 +122,11 @@ struct DecodeCfg {
     static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 2));
     static constexpr int MERGE_BYTES = HKV * (KSPLIT - 1) * MERGE_FLOATS_PER_WARP * 4;
     static constexpr int PLAN_BYTES = (kMaxRegions + 2) * 4;
+    // ring depth: what fits beside the merge buffer and the plan in the 227 KB a CTA may use (3 KB are
+    // left for static shared memory and the 1 KB alignment slack), at most 4 stages
+    static constexpr int FIT = (232448 - 3072 - 1024 - MERGE_BYTES - PLAN_BYTES - 256) / STAGE_BYTES;
+    static constexpr int NSTAGE = FIT > 4 ? 4 : FIT;
+    static_assert(NSTAGE >= 2, "decode pipeline needs two stages");
     static constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + MERGE_BYTES + PLAN_BYTES + 256;
 };
 
@@ -391,11 +396,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
             // ---- online softmax (exp2 domain) ----
             const bool tail = j0 + 16 > len;
-            uint32_t pa[4];
+            uint32_t pa[4], pb[4];  // P = pa + pb: bf16 head and bf16 remainder of every probability
             float corr[2];
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
-                if (i >= NROW) { pa[i] = 0u; pa[i + 2] = 0u; corr[i] = 1.f; continue; }
+                if (i >= NROW) { pa[i] = pa[i + 2] = pb[i] = pb[i + 2] = 0u; corr[i] = 1.f; continue; }
                 float x[4];
                 x[0] = sacc[0][2 * i] * p.sl2; x[1] = sacc[0][2 * i + 1] * p.sl2;
                 x[2] = sacc[1][2 * i] * p.sl2; x[3] = sacc[1][2 * i + 1] * p.sl2;
@@ -412,10 +417,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const float mn = fmaxf(m_run[i], mx);  // finite: row j0 of the block is valid
                 corr[i] = exp2_or_zero(m_run[i], mn);
                 m_run[i] = mn;
-                pa[i] = pack_bf16(fast_exp2(x[0] - mn), fast_exp2(x[1] - mn));
-                pa[i + 2] = pack_bf16(fast_exp2(x[2] - mn), fast_exp2(x[3] - mn));
-                // the row sum uses the bf16-rounded probabilities the PV product sees
-                l_run[i] = l_run[i] * corr[i] + ((bf16lo(pa[i]) + bf16hi(pa[i])) + (bf16lo(pa[i + 2]) + bf16hi(pa[i + 2])));
+                const float e0 = fast_exp2(x[0] - mn), e1 = fast_exp2(x[1] - mn);
+                const float e2 = fast_exp2(x[2] - mn), e3 = fast_exp2(x[3] - mn);
+                pa[i] = pack_bf16(e0, e1);
+                pa[i + 2] = pack_bf16(e2, e3);
+                pb[i] = pack_bf16(e0 - bf16lo(pa[i]), e1 - bf16hi(pa[i]));
+                pb[i + 2] = pack_bf16(e2 - bf16lo(pa[i + 2]), e3 - bf16hi(pa[i + 2]));
+                l_run[i] = l_run[i] * corr[i] + ((e0 + e1) + (e2 + e3));
             }
             if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
@@ -444,6 +452,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     if (tail) { b[0] &= vmask0; b[1] &= vmask1; b[2] &= vmask0; b[3] &= vmask1; }
                     mma_bf16_16816(oacc[2 * n2], pa[0], pa[1], pa[2], pa[3], b[0], b[1]);
                     mma_bf16_16816(oacc[2 * n2 + 1], pa[0], pa[1], pa[2], pa[3], b[2], b[3]);
+                    mma_bf16_16816(oacc[2 * n2], pb[0], pb[1], pb[2], pb[3], b[0], b[1]);
+                    mma_bf16_16816(oacc[2 * n2 + 1], pb[0], pb[1], pb[2], pb[3], b[2], b[3]);
                 }
             }
         }
