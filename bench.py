@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of the AirCache compress-then-decode hot path on B200.
+
+One *step* is one pass of the whole path over one batch of synthetic requests: for every resident request
+the compression (aircache_score -> aircache_budget -> aircache_compact over all layers), then `decode_steps`
+rounds of single-token decode attention (aircache_decode_attn over all layers) with a fresh query per round.
+`rotate` independent requests (different seeds) are resident and are served round-robin, so that consecutive
+decode launches never find their cache in L2: the per-launch working set of one request at 10 % retention
+(49 MB) is smaller than the 126 MB L2, the rotation makes every launch read HBM as it would between the
+layers of a real model.
+
+  value           tokens / s over the whole step (compression included), inputs resident in HBM
+  decode_tok_s    tokens / s over the decode region of the step alone
+  compress_us_per_layer   (score + budget + compact) / layers, per request
+  roofline        decode attention: algorithmic bytes (every valid K' and V' row once, q and output) per
+                  call / average duration of a call inside the timed region
+  e2e             the same metric through aircache_pipeline_host: pinned host inputs, host outputs
+  cpu_baseline    the CPU oracle timed on this host (rank 0, N = 1 only)
+
+`python bench.py --impl reference` times the CPU oracle instead (there is no other implementation of the
+paper's method to run).  Under torchrun every rank runs the same workload on its own GPU with its own seeds
+(no data-path collective: requests are independent); times are device times, maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "decode_tok_s_at_10pct_visual_kv"
+UNIT = "tok/s"
+L2_BYTES = 126 * 2 ** 20
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from the ncu capture summarised
+# in profiles/; valid only for the kernel source it was taken on (sha1 of csrc/decode.cu, first 12 hex).
+NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "", "bytes_per_launch": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2", help="c1 | c2 | c3[:batch] | c4 | c5")
+    ap.add_argument("--ratio", type=float, default=None)
+    ap.add_argument("--rotate", type=int, default=0, help="resident requests (0 = enough to exceed 2x L2)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="decode rounds per step (0 = the workload's)")
+    ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def pick_workload(spec: str, ratio):
+    from workloads import CONFIGS
+    name, _, arg = spec.partition(":")
+    wl = CONFIGS[name]
+    if arg:
+        wl = wl.with_(batch=int(arg))
+    if ratio is not None:
+        wl = wl.with_(ratio=ratio)
+    return wl
+
+
+def shape_of(ac, wl):
+    return ac.shape(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_visual, wl.n_text,
+                    wl.window, wl.slack, wl.scale)
+
+
+def logical(t):
+    return t.permute(0, 1, 3, 2, 4)
+
+
+# --------------------------------------------------------------------------------------------------
+# distributed plumbing (one process per GPU; gloo on CPU in the tests)
+# --------------------------------------------------------------------------------------------------
+def dist_info():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_over_ranks(local_ms: float, local_units: float, device, dist=None):
+    """(max over ranks of the time, sum over ranks of the units).  Works with any backend."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms, local_units
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def decode_cu_sha1():
+    p = os.path.join(ROOT, "paper_2503_23956_b200", "csrc", "decode.cu")
+    return hashlib.sha1(open(p, "rb").read()).hexdigest()[:12]
+
+
+def run_cuda(args):
+    import paper_2503_23956_b200 as ac
+    from paper_2503_23956_b200.session import Session
+    from workloads import decode_queries, full_cache, window_queries
+
+    rank, local_rank, world = dist_info()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the AirCache path has no CPU fallback")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    ac.lib()  # fail loudly if the library is missing
+
+    wl = pick_workload(args.workload, args.ratio)
+    n_dec = args.decode_steps or wl.steps
+    sh = shape_of(ac, wl)
+    row_bytes = wl.n_kv_heads * wl.head_dim * 2
+    T = ac.aircache_kept_per_sequence(sh, wl.ratio)
+    cache_bytes = 2 * row_bytes * wl.batch * (T + wl.n_layers * wl.n_text)   # K' + V' valid rows of one request batch
+    rotate = args.rotate or max(2, -(-2 * L2_BYTES // cache_bytes))
+    rotate = min(rotate, 16)
+
+    # ---- resident inputs: `rotate` independent request batches ----
+    reqs = []
+    for i in range(rotate):
+        w = wl.with_(seed=wl.seed + 1000 * rank + i)
+        s = Session(sh, wl.ratio, wl.alpha, dev)
+        k, v = full_cache(w, "k", dev), full_cache(w, "v", dev)
+        s.set_full(logical(k), logical(v))
+        s.qw = window_queries(w, dev)
+        s.q_steps = torch.stack([decode_queries(w, t, dev) for t in range(n_dec)]).contiguous()
+        s.out_steps = torch.empty((n_dec,) + tuple(s.out.shape), dtype=torch.float32, device=dev)
+        reqs.append(s)
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.Stream(device=dev)
+    launches = {"score": 3, "budget": 2, "compact": 2, "decode": 2}   # kernels per C-ABI call
+
+    def stage_score():
+        for s in reqs:
+            s.score(s.qw, stream=stream)
+
+    def stage_budget():
+        for s in reqs:
+            s.budget(stream=stream)
+
+    def stage_compact():
+        for s in reqs:
+            s.compact(want_kept=False, stream=stream)
+
+    def stage_decode():
+        for t in range(n_dec):
+            for s in reqs:
+                s.decode(s.q_steps[t], out=s.out_steps[t], stream=stream)
+
+    stages = [("score", stage_score), ("budget", stage_budget), ("compact", stage_compact), ("decode", stage_decode)]
+    graphs = {}
+    with torch.cuda.stream(stream):
+        for _, fn in stages[:3]:
+            fn()       # one eager pass: the compressed caches exist before the decode graph is captured
+        stream.synchronize()
+        if not args.no_graph:
+            for name, fn in stages:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    fn()
+                graphs[name] = g
+
+    def run_step(ev):
+        ev[0].record(stream)
+        for i, (name, fn) in enumerate(stages):
+            if graphs:
+                graphs[name].replay()
+            else:
+                fn()
+            ev[i + 1].record(stream)
+
+    def new_events():
+        return [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            run_step(new_events())
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank)
+        evs = [new_events() for _ in range(args.steps)]
+        for e in evs:
+            run_step(e)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        clocks = sampler.stop()
+    for s in reqs:
+        if s.status() != 0:
+            raise RuntimeError("a device-side wait timed out")
+
+    total_ms = evs[0][0].elapsed_time(evs[-1][4])
+    stage_ms = {name: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / args.steps
+                for i, (name, _) in enumerate(stages)}
+    tokens_per_step = rotate * n_dec * wl.batch
+    total_ms_all, tokens_all = reduce_over_ranks(total_ms, tokens_per_step * args.steps, dev, dist)
+    decode_ms_all, _ = reduce_over_ranks(stage_ms["decode"], 0, dev, dist)
+
+    # ---- roofline of the dominant kernel (decode attention) ----
+    valid_rows = sum(int(s.lens.sum().item()) for s in reqs) / rotate
+    q_out_bytes = wl.n_layers * wl.batch * wl.n_q_heads * wl.head_dim * 6
+    alg_bytes = 2 * row_bytes * valid_rows + q_out_bytes
+    calls = rotate * n_dec
+    call_us = stage_ms["decode"] * 1e3 / calls
+    achieved = alg_bytes / (call_us * 1e-6) / 1e9
+    peak, peak_kind = measured_peaks()
+    traffic = None
+    if NCU_TRAFFIC["bytes_per_launch"] and NCU_TRAFFIC["decode_cu_sha1"] == decode_cu_sha1() \
+            and NCU_TRAFFIC["workload"] == args.workload and args.ratio is None:
+        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    compact_bytes = 2 * alg_bytes - 2 * q_out_bytes + 4 * wl.batch * T     # read + write of every kept row, indices
+    comp_us = stage_ms["compact"] * 1e3 / rotate
+
+    result = {
+        "metric": METRIC, "value": tokens_all / (total_ms_all * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms_all / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name} r={wl.ratio:g} B={wl.batch} L={wl.n_layers} Hq={wl.n_q_heads} "
+                               f"Hkv={wl.n_kv_heads} d={wl.head_dim} Nv={wl.n_visual} Nt={wl.n_text} W={wl.window}",
+                   "decode_steps": n_dec, "resident_requests": rotate,
+                   "l2": f"inputs larger than L2: {rotate} independent requests served round-robin, "
+                         f"{rotate * cache_bytes / 2 ** 20:.0f} MiB of compressed cache cycled per decode round",
+                   "launch": "CUDA graph replay of the C-ABI calls" if graphs else "direct C-ABI calls",
+                   "attention_only": True},
+        "decode_tok_s": world * tokens_per_step / (decode_ms_all * 1e-3),
+        "compress_us_per_layer": (stage_ms["score"] + stage_ms["budget"] + stage_ms["compact"]) * 1e3
+                                 / (rotate * wl.n_layers),
+        "stage_us_per_request": {k: v * 1e3 / rotate for k, v in stage_ms.items()},
+        "roofline": {"kernel": "decode_kernel (+combine_kernel) per aircache_decode_attn call", "bound": "hbm",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
+                     "bytes_per_call": alg_bytes, "us_per_call": call_us},
+        "roofline_compact": {"kernel": "select_kernel + gather_kernel per aircache_compact call", "bound": "hbm",
+                             "achieved": compact_bytes / (comp_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                             "frac": compact_bytes / (comp_us * 1e-6) / 1e9 / peak, "bytes_per_call": compact_bytes,
+                             "us_per_call": comp_us},
+        "clocks": clocks,
+        "gpu_launches": args.steps * rotate * (launches["score"] + launches["budget"] + launches["compact"]
+                                               + n_dec * launches["decode"]),
+    }
+
+    if rank == 0 and not args.no_e2e:
+        result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 5))
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(wl, n_dec)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
+    """Same metric through aircache_pipeline_host: every step uploads the full cache and the queries from
+    pinned host memory, runs the whole path and downloads the attention outputs and the budgets."""
+    stream = torch.cuda.current_stream(dev)
+    k_tm = s.k_full.permute(0, 1, 3, 2, 4)      # back to the token-major storage order
+    v_tm = s.v_full.permute(0, 1, 3, 2, 4)
+    assert k_tm.is_contiguous()
+    h_k, h_v = k_tm.cpu().pin_memory(), v_tm.cpu().pin_memory()
+    h_full = ac.full_view(logical(h_k), logical(h_v))
+    d_k, d_v = torch.empty_like(k_tm), torch.empty_like(v_tm)
+    h_qw, h_q = s.qw.cpu().pin_memory(), s.q_steps.cpu().pin_memory()
+    d_qw, d_q = torch.empty_like(s.qw), torch.empty_like(s.q_steps)
+    h_out = torch.empty(s.out_steps.shape, dtype=torch.float32).pin_memory()
+    h_bud = torch.empty(s.budgets.shape, dtype=torch.int32).pin_memory()
+
+    def once():
+        ac.aircache_pipeline_host(sh, h_full, h_k.numel(), d_k, d_v, h_qw, d_qw, h_q, d_q, n_dec, wl.alpha,
+                                  wl.ratio, 0, s.scores, s.budgets, s.cache, s.out_steps, h_out, h_bud, s.ws, stream)
+
+    once()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        once()      # synchronises internally after the device-to-host copies
+    dt = (time.perf_counter() - t0) / steps
+    h2d = 2 * h_k.numel() * 2 + h_qw.numel() * 2 + h_q.numel() * 2
+    d2h = h_out.numel() * 4 + h_bud.numel() * 4
+    return {"value": n_dec * wl.batch / dt, "unit": UNIT, "ms_per_step": dt * 1e3, "requests_per_step": 1,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "aircache_pipeline_host"}
+
+
+# --------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(wl, n_dec, max_seqs=1, dec_rounds=4):
+    """Times the oracle on a bounded sample of the workload: the whole compression of `max_seqs` sequences
+    (all layers) and `dec_rounds` decode rounds over their compressed caches; returns seconds."""
+    import oracle
+    from workloads import decode_queries, full_cache, window_queries
+    from workloads.synth import to_u16
+    oracle.build()
+    seqs = list(range(min(max_seqs, wl.batch)))
+    w1 = wl.with_(batch=len(seqs))
+    dm = oracle.Dims(w1.n_layers, w1.batch, w1.n_q_heads, w1.n_kv_heads, w1.head_dim, w1.n_visual, w1.n_text,
+                     w1.window)
+    k, v = full_cache(wl, "k", "cpu", seqs=seqs), full_cache(wl, "v", "cpu", seqs=seqs)
+    qw = window_queries(wl, "cpu", seqs=seqs)
+    kl, vl = to_u16(k).transpose(0, 1, 3, 2, 4), to_u16(v).transpose(0, 1, 3, 2, 4)
+    t0 = time.perf_counter()
+    sc = oracle.score(dm, kl, to_u16(qw), wl.scale, wl.alpha)
+    st, sk = oracle.moments(sc["scores"])
+    bud = oracle.allocate(st, sk, wl.n_visual, wl.ratio, 0)
+    cp = oracle.compact(dm, 0, kl, vl, sc["scores"], bud)
+    t_comp = time.perf_counter() - t0
+    qs = [to_u16(decode_queries(wl, t, "cpu", seqs=seqs)) for t in range(dec_rounds)]
+    t0 = time.perf_counter()
+    for q in qs:
+        oracle.decode(dm, cp["k"], cp["v"], cp["offsets"], cp["lens"], q, wl.scale)
+    t_dec = (time.perf_counter() - t0) / dec_rounds
+    # scale to the whole batch: sequences are independent, the oracle's cost is linear in them
+    f = wl.batch / len(seqs)
+    return {"t_compress": t_comp * f, "t_decode_round": t_dec * f, "threads": oracle.num_threads(),
+            "sample": f"oracle on {len(seqs)} of {wl.batch} sequence(s), all {wl.n_layers} layers: whole compression "
+                      f"once + {dec_rounds} decode rounds; scaled linearly to the batch and to {n_dec} rounds"}
+
+
+def cpu_baseline(wl, n_dec):
+    s = oracle_sample(wl, n_dec)
+    step_s = s["t_compress"] + n_dec * s["t_decode_round"]
+    return {"value": n_dec * wl.batch / step_s, "unit": UNIT, "cores": s["threads"], "kind": "oracle",
+            "sample": s["sample"], "compress_us_per_layer": s["t_compress"] * 1e6 / (wl.n_layers * wl.batch),
+            "decode_tok_s": wl.batch / s["t_decode_round"]}
+
+
+def run_reference(args):
+    rank, _, world = dist_info()
+    if rank != 0:
+        return
+    wl = pick_workload(args.workload, args.ratio)
+    n_dec = args.decode_steps or wl.steps
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(wl, n_dec, dec_rounds=1)
+    times, last = [], None
+    for _ in range(args.steps):
+        last = oracle_sample(wl, n_dec, dec_rounds=2)
+        times.append(last["t_compress"] + n_dec * last["t_decode_round"])
+    step_s = sum(times) / len(times)
+    value = n_dec * wl.batch / step_s
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name} r={wl.ratio:g} B={wl.batch} L={wl.n_layers} Hq={wl.n_q_heads} "
+                               f"Hkv={wl.n_kv_heads} d={wl.head_dim} Nv={wl.n_visual} Nt={wl.n_text} W={wl.window}",
+                   "decode_steps": n_dec, "attention_only": True},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["threads"], "kind": "oracle",
+                         "sample": last["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_cuda(a)

@@ -60,6 +60,7 @@ WsLayout ws_layout(const aircache_shape_t *s) {
         return at;
     };
     w.status = take(256);
+    w.tickets = take((int64_t)kMaxRegions * 4);
     w.row_count = take(groups * 4);
     w.row_info = take(groups * cap * 4);
     w.row_coef = take(groups * cap * 4);
@@ -71,7 +72,6 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.alloc_share = take(LB * 8);
     w.alloc_active = take(LB * 4);
     w.kept = take(LB * s->n_visual * 4);
-    w.plan = take((LB + 2) * 4);
     w.partials = take((int64_t)2 * kMaxDecodeCtas * s->n_q_heads * (s->head_dim + 2) * 4);
     w.total = off;
     return w;
@@ -211,8 +211,8 @@ int aircache_append(const aircache_shape_t *shape, aircache_ragged_t *cache, con
 int aircache_reset_status(void *workspace, int64_t workspace_bytes, void *cuda_stream) {
     if (!workspace) return AIRCACHE_ERR_INVALID_ARG;
     if ((uintptr_t)workspace & 255) return AIRCACHE_ERR_ALIGNMENT;
-    if (workspace_bytes < 256) return AIRCACHE_ERR_WORKSPACE_TOO_SMALL;
-    AIRCACHE_CUDA_TRY(cudaMemsetAsync(workspace, 0, 256, (cudaStream_t)cuda_stream));
+    if (workspace_bytes < kStatusBytes) return AIRCACHE_ERR_WORKSPACE_TOO_SMALL;
+    AIRCACHE_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)cuda_stream));
     return AIRCACHE_OK;
 }
 

@@ -15,6 +15,7 @@ constexpr int kMaxRegions = 2048;     // L * B (the decode kernel keeps the unit
 constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int64_t kStatusBytes = 256 + (int64_t)kMaxRegions * 4;  // status word + tickets, at the start of the workspace
 
 // ---------------------------------------------------------------------------------------------
 // error plumbing
@@ -67,6 +68,7 @@ inline int score_chunks(const aircache_shape_t *s) {
 
 struct WsLayout {
     int64_t status;       // u32 status word (256 bytes reserved)
+    int64_t tickets;      // i32  [kMaxRegions]        split-K tickets of the decode kernel, zero between calls
     int64_t row_count;    // i32  [L*B*Hkv]            elite rows of the KV group
     int64_t row_info;     // i32  [L*B*Hkv][cap]       (head within group << 8) | window slot
     int64_t row_coef;     // f32  [L*B*Hkv][cap]       1 / (|E_h| * Hq)
@@ -78,7 +80,6 @@ struct WsLayout {
     int64_t alloc_share;  // f64  [L*B]
     int64_t alloc_active; // i32  [L*B]
     int64_t kept;         // i32  [L*B*Nv]             kept-token lists when the caller passes none
-    int64_t plan;         // i32  [L*B + 2]            unit prefix of the decode schedule (+ total)
     int64_t partials;     // f32  [2*kMaxDecodeCtas][Hq*(d+2)]
     int64_t total;
 };

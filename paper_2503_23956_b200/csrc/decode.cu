@@ -1,5 +1,5 @@
 // aircache_decode_attn: single-token attention over the ragged compressed cache (Section 3.1, token
-// decoding), all layers and sequences in one persistent launch plus a small combine launch.
+// decoding), all layers and sequences in one persistent launch.
 //
 // Work decomposition.  A "unit" is CH consecutive rows of one region (all KV heads, K and V).  Region r
 // has ceil(lens[r] / CH) units; every CTA first scans these counts into a prefix P (shared memory), then
@@ -7,7 +7,9 @@
 // The load is therefore balanced to one unit regardless of how ragged the regions are.  Consecutive units
 // of one region accumulate in registers; a region that lies wholly inside one CTA's range is finished and
 // written by that CTA, otherwise the CTA writes an unnormalised partial (running max, sum, accumulator) and
-// combine_kernel merges the partials of the region in CTA order (split-K, fixed order).
+// takes a ticket of the region; the CTA that draws the last ticket merges the region's partials in CTA
+// order (split-K with a fixed combination order, whoever arrives last) and puts the ticket back to zero
+// for the next call.  Nobody waits for anybody.
 //
 // Inside a CTA.  One producer warp streams units through a ring of shared-memory stages with TMA
 // (cp.async.bulk.tensor, 128-byte swizzle, one box of CH rows x 64 channels per KV head and half of
@@ -39,7 +41,7 @@ struct DecodeParams {
     float *out;              // [L*B, Hq, D]
     const int64_t *offsets;  // [L*B + 1]
     const int32_t *lens;     // [L*B]
-    int32_t *plan;           // [L*B + 2] unit prefix written by CTA 0 for the combine kernel
+    int32_t *tickets;        // [L*B] partials of the region written so far; zero between calls
     float *partials;         // [2 * CTAs][Hq * (D + 2)]
     uint32_t *status;
     int n_regions, Hq, G;
@@ -154,6 +156,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + kStages * C::STAGE_BYTES + C::MERGE_BYTES + C::PLAN_BYTES);
     __shared__ int s_part[C::THREADS];
     __shared__ int s_abort;
+    __shared__ int s_last;
 
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int n = p.n_regions;
@@ -205,8 +208,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         __syncthreads();
     }
     const int total = s_P[n];
-    if (blockIdx.x == 0) {
-        for (int i = tid; i <= n; i += C::THREADS) p.plan[i] = s_P[i];
+    // a region without rows yields zeros
+    for (int r = blockIdx.x; r < n; r += gridDim.x) {
+        if (s_P[r + 1] == s_P[r])
+            for (int i = tid; i < p.Hq * D; i += C::THREADS) p.out[(int64_t)r * p.Hq * D + i] = 0.f;
     }
     const int upc = max(1, (total + (int)gridDim.x - 1) / (int)gridDim.x);
     const int u0 = min(total, (int)blockIdx.x * upc), u1 = min(total, u0 + upc);
@@ -326,8 +331,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
             consumer_bar(NCW * 32);
         }
+        const bool whole = (ustart == s_P[r]) && (uend == s_P[r + 1]);
         if (ks == 0) {
-            const bool whole = (ustart == s_P[r]) && (uend == s_P[r + 1]);
 #pragma unroll
             for (int i = 0; i < NROW; ++i) {
                 const int hl = gid + 8 * i;
@@ -346,11 +351,52 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     float *o = base + (size_t)h * D;
 #pragma unroll
                     for (int nd = 0; nd < D / 8; ++nd)
-                        *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) = make_float2(oacc[nd][2 * i], oacc[nd][2 * i + 1]);
+                        __stcg(reinterpret_cast<float2 *>(o + nd * 8 + 2 * t),
+                               make_float2(oacc[nd][2 * i], oacc[nd][2 * i + 1]));
                     if (t == 0) {
-                        base[(size_t)p.Hq * D + h] = m_run[i];
-                        base[(size_t)p.Hq * (D + 1) + h] = l_run[i];
+                        __stcg(base + (size_t)p.Hq * D + h, m_run[i]);
+                        __stcg(base + (size_t)p.Hq * (D + 1) + h, l_run[i]);
                     }
+                }
+            }
+        }
+        if (!whole) {
+            // split-K combine without a second launch: publish the partial, draw a ticket; the CTA that draws
+            // the region's last ticket merges all partials in CTA order
+            __threadfence();
+            consumer_bar(NCW * 32);
+            const int c0 = s_P[r] / upc, c1 = (s_P[r + 1] - 1) / upc;
+            if (tid == 0) {
+                const int tk = atomicAdd(p.tickets + r, 1);
+                s_last = (tk == c1 - c0);
+                if (s_last) p.tickets[r] = 0;
+                __threadfence();
+            }
+            consumer_bar(NCW * 32);
+            if (s_last) {
+                const size_t slot_floats = (size_t)p.Hq * (D + 2);
+                const int P0 = s_P[r];
+                for (int i = tid; i < p.Hq * D / 4; i += NCW * 32) {
+                    const int h = (i * 4) / D;
+                    float m_tot = -INFINITY;
+                    for (int c = c0; c <= c1; ++c) {
+                        const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
+                        m_tot = fmaxf(m_tot, __ldcg(p.partials + slot * slot_floats + (size_t)p.Hq * D + h));
+                    }
+                    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float den = 0.f;
+#pragma unroll 4
+                    for (int c = c0; c <= c1; ++c) {
+                        const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
+                        const float *base = p.partials + slot * slot_floats;
+                        const float w = exp2_or_zero(__ldcg(base + (size_t)p.Hq * D + h), m_tot);
+                        const float4 a = __ldcg(reinterpret_cast<const float4 *>(base) + i);
+                        num.x += a.x * w; num.y += a.y * w; num.z += a.z * w; num.w += a.w * w;
+                        den += __ldcg(base + (size_t)p.Hq * (D + 1) + h) * w;
+                    }
+                    const float inv = den > 0.f ? 1.0f / den : 0.f;
+                    reinterpret_cast<float4 *>(p.out + (int64_t)r * p.Hq * D)[i] =
+                        make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
                 }
             }
         }
@@ -463,40 +509,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     if (ok) flush(r, seg_start, u1);
 }
 
-// Merges the partials of every region that more than one CTA worked on.  grid = regions, 128 threads.
-template <int D>
-__global__ void __launch_bounds__(128) combine_kernel(DecodeParams p, int n_ctas) {
-    const int r = blockIdx.x;
-    const int n = p.n_regions;
-    const int P0 = p.plan[r], P1 = p.plan[r + 1], total = p.plan[n];
-    float *o = p.out + (int64_t)r * p.Hq * D;
-    if (P1 == P0) {
-        for (int i = threadIdx.x; i < p.Hq * D; i += blockDim.x) o[i] = 0.f;
-        return;
-    }
-    const int upc = max(1, (total + n_ctas - 1) / n_ctas);
-    const int c0 = P0 / upc, c1 = (P1 - 1) / upc;
-    if (c0 == c1) return;  // finished inside the decode kernel
-    const size_t slot_floats = (size_t)p.Hq * (D + 2);
-    for (int i = threadIdx.x; i < p.Hq * D; i += blockDim.x) {
-        const int h = i / D;
-        float m_tot = -INFINITY;
-        for (int c = c0; c <= c1; ++c) {
-            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
-            m_tot = fmaxf(m_tot, p.partials[slot * slot_floats + (size_t)p.Hq * D + h]);
-        }
-        float num = 0.f, den = 0.f;
-        for (int c = c0; c <= c1; ++c) {
-            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
-            const float *base = p.partials + slot * slot_floats;
-            const float w = exp2_or_zero(base[(size_t)p.Hq * D + h], m_tot);
-            num += base[i] * w;
-            den += base[(size_t)p.Hq * (D + 1) + h] * w;
-        }
-        o[i] = den > 0.f ? num / den : 0.f;
-    }
-}
-
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
@@ -552,8 +564,6 @@ int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st
                                            C::SMEM_BYTES));
     decode_kernel<D, HKV, G_HI><<<ctas, C::THREADS, C::SMEM_BYTES, st>>>(tm_k, tm_v, p);
     AIRCACHE_LAUNCH_CHECK();
-    combine_kernel<D><<<p.n_regions, 128, 0, st>>>(p, ctas);
-    AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }
 
@@ -583,7 +593,7 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.out = out;
     p.offsets = c->offsets;
     p.lens = c->lens;
-    p.plan = ws_ptr<int32_t>(ws, w.plan);
+    p.tickets = ws_ptr<int32_t>(ws, w.tickets);
     p.partials = ws_ptr<float>(ws, w.partials);
     p.status = ws_ptr<uint32_t>(ws, w.status);
     p.n_regions = s->n_layers * s->batch;

@@ -6,6 +6,7 @@ import numpy as np
 import torch
 
 import paper_2503_23956_b200 as ac
+from paper_2503_23956_b200.session import Session
 from workloads import decode_queries, full_cache, window_queries
 from workloads.synth import to_u16
 
@@ -40,57 +41,13 @@ def u16(t: torch.Tensor) -> np.ndarray:
     return to_u16(t)
 
 
-class GpuPath:
+class GpuPath(Session):
     """Device buffers of one workload and the four stages as methods (thin calls into the C ABI)."""
 
     def __init__(self, wl, ratio=None, device="cuda:0", slack=None):
         self.wl = wl
-        self.dev = torch.device(device)
-        self.ratio = wl.ratio if ratio is None else ratio
         self.slack = wl.slack if slack is None else slack
-        self.sh = shape_of(wl, slack=self.slack)
-        LB = wl.n_layers * wl.batch
-        self.ws = torch.empty(ac.aircache_workspace_bytes(self.sh), dtype=torch.uint8, device=self.dev)
-        ac.aircache_reset_status(self.ws)
-        self.scores = torch.empty((wl.n_layers, wl.batch, wl.n_visual), dtype=torch.float32, device=self.dev)
-        self.mask = torch.zeros((wl.n_layers, wl.batch, wl.n_q_heads), dtype=torch.int64, device=self.dev)
-        self.budgets = torch.empty((wl.n_layers, wl.batch), dtype=torch.int32, device=self.dev)
-        self.strength = torch.empty((wl.n_layers, wl.batch), dtype=torch.float64, device=self.dev)
-        self.skew = torch.empty((wl.n_layers, wl.batch), dtype=torch.float64, device=self.dev)
-        self.rows = ac.aircache_total_rows(self.sh, self.ratio)
-        self.kept_n = wl.batch * ac.aircache_kept_per_sequence(self.sh, self.ratio)
-        self.k_c = torch.empty((self.rows, wl.n_kv_heads, wl.head_dim), dtype=torch.bfloat16, device=self.dev)
-        self.v_c = torch.empty_like(self.k_c)
-        self.offsets = torch.zeros(LB + 1, dtype=torch.int64, device=self.dev)
-        self.lens = torch.zeros(LB, dtype=torch.int32, device=self.dev)
-        self.kept = torch.empty(max(self.kept_n, 1), dtype=torch.int32, device=self.dev)
-        self.cache = ac.ragged_view(self.k_c, self.v_c, self.offsets, self.lens, self.rows)
-        self.out = torch.empty((wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32,
-                               device=self.dev)
-
-    def set_full(self, k_log: torch.Tensor, v_log: torch.Tensor):
-        """k_log, v_log: device bf16 tensors with logical dims [L,B,Hkv,N,d]."""
-        self.k_full, self.v_full = k_log, v_log
-        self.full = ac.full_view(k_log, v_log)
-
-    def score(self, qw, alpha=None):
-        ac.aircache_score(self.sh, self.full, qw, self.wl.alpha if alpha is None else alpha, self.scores, self.mask,
-                          self.ws)
-
-    def budget(self, scores=None, mode=0):
-        ac.aircache_budget(self.sh, self.scores if scores is None else scores, self.ratio, mode, self.budgets,
-                           self.strength, self.skew, self.cache, self.ws)
-
-    def compact(self, scores=None, budgets=None, want_kept=True):
-        ac.aircache_compact(self.sh, self.full, self.scores if scores is None else scores,
-                            self.budgets if budgets is None else budgets, self.ratio, self.cache,
-                            self.kept if want_kept else None, self.ws)
-
-    def decode(self, q, out=None):
-        ac.aircache_decode_attn(self.sh, self.cache, q, self.out if out is None else out, self.ws)
-
-    def status(self):
-        return ac.aircache_check_status(self.ws, check=False)
+        super().__init__(shape_of(wl, slack=self.slack), wl.ratio if ratio is None else ratio, wl.alpha, device)
 
 
 def gen_inputs(wl, device):
