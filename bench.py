@@ -204,7 +204,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
 
     stream = torch.cuda.Stream(device=dev)
-    launches = {"score": 3, "budget": 2, "compact": 2, "decode": 2}   # kernels per C-ABI call
+    launches = {"score": 3, "budget": 2, "compact": 2, "decode": 1}   # kernels per C-ABI call
 
     def stage_score():
         for s in reqs:
@@ -304,7 +304,7 @@ def run_cuda(args):
         "compress_us_per_layer": (stage_ms["score"] + stage_ms["budget"] + stage_ms["compact"]) * 1e3
                                  / (rotate * wl.n_layers),
         "stage_us_per_request": {k: v * 1e3 / rotate for k, v in stage_ms.items()},
-        "roofline": {"kernel": "decode_kernel (+combine_kernel) per aircache_decode_attn call", "bound": "hbm",
+        "roofline": {"kernel": "decode_kernel (one launch per aircache_decode_attn call)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
                      "bytes_per_call": alg_bytes, "us_per_call": call_us},

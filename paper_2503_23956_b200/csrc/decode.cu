@@ -376,23 +376,40 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             if (s_last) {
                 const size_t slot_floats = (size_t)p.Hq * (D + 2);
                 const int P0 = s_P[r];
+                // every thread owns float4 columns of the [Hq, D] result; the partials are visited eight at a
+                // time with all their loads in flight together, merged online in CTA order
                 for (int i = tid; i < p.Hq * D / 4; i += NCW * 32) {
                     const int h = (i * 4) / D;
-                    float m_tot = -INFINITY;
-                    for (int c = c0; c <= c1; ++c) {
-                        const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
-                        m_tot = fmaxf(m_tot, __ldcg(p.partials + slot * slot_floats + (size_t)p.Hq * D + h));
-                    }
+                    float M = -INFINITY, den = 0.f;
                     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-                    float den = 0.f;
-#pragma unroll 4
-                    for (int c = c0; c <= c1; ++c) {
-                        const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
-                        const float *base = p.partials + slot * slot_floats;
-                        const float w = exp2_or_zero(__ldcg(base + (size_t)p.Hq * D + h), m_tot);
-                        const float4 a = __ldcg(reinterpret_cast<const float4 *>(base) + i);
-                        num.x += a.x * w; num.y += a.y * w; num.z += a.z * w; num.w += a.w * w;
-                        den += __ldcg(base + (size_t)p.Hq * (D + 1) + h) * w;
+                    for (int cb = c0; cb <= c1; cb += 8) {
+                        float mm[8], ll[8];
+                        float4 aa[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int c = min(cb + j, c1);
+                            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
+                            const float *base = p.partials + slot * slot_floats;
+                            mm[j] = __ldcg(base + (size_t)p.Hq * D + h);
+                            ll[j] = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
+                            aa[j] = __ldcg(reinterpret_cast<const float4 *>(base) + i);
+                        }
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (cb + j > c1) mm[j] = -INFINITY;
+                            mx = fmaxf(mx, mm[j]);
+                        }
+                        const float Mn = fmaxf(M, mx);
+                        const float sc = exp2_or_zero(M, Mn);
+                        num.x *= sc; num.y *= sc; num.z *= sc; num.w *= sc; den *= sc;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float w = exp2_or_zero(mm[j], Mn);
+                            num.x += aa[j].x * w; num.y += aa[j].y * w; num.z += aa[j].z * w; num.w += aa[j].w * w;
+                            den += ll[j] * w;
+                        }
+                        M = Mn;
                     }
                     const float inv = den > 0.f ? 1.0f / den : 0.f;
                     reinterpret_cast<float4 *>(p.out + (int64_t)r * p.Hq * D)[i] =
