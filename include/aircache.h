@@ -55,6 +55,10 @@ extern "C" {
 #define AIRCACHE_ERR_CAPACITY (-5)             /* ragged cache smaller than aircache_total_rows()               */
 #define AIRCACHE_ERR_CUDA (-6)                 /* a CUDA call failed; see aircache_last_cuda_error()            */
 #define AIRCACHE_ERR_TIMEOUT (-7)              /* a bounded device-side wait gave up (aircache_check_status)    */
+#define AIRCACHE_ERR_STATIC_SCRATCH (-8)       /* aircache_decode_attn_static: built-in scratch array too small */
+
+/* Size of the device array that aircache_decode_attn_static uses as scratch, per GPU. */
+#define AIRCACHE_STATIC_SCRATCH_BYTES (12 * 1024 * 1024)
 
 /* Problem shape, uniform over the batch. */
 typedef struct {
@@ -183,6 +187,39 @@ int aircache_compact(const aircache_shape_t *shape, const aircache_full_t *full,
  */
 int aircache_decode_attn(const aircache_shape_t *shape, const aircache_ragged_t *cache, const void *q,
                          float *out, void *workspace, int64_t workspace_bytes, void *cuda_stream);
+
+/*
+ * aircache_decode_attn for callers that cannot allocate device memory.  (An
+ * addition of this library; the paper has no counterpart.)
+ *
+ * Some hosts of this code only ever borrow the GPU: a plug-in running inside
+ * another engine's memory pool, a real-time loop that may not enter the
+ * allocator after start-up, a process whose device memory is fully
+ * pre-assigned.  They can hand over the cache, the query and the output, but
+ * have nowhere to get the workspace that aircache_decode_attn wants.  This
+ * entry point runs the same kernel and takes the kernel's scratch (status
+ * word, split-K tickets, partial results) from an array of
+ * AIRCACHE_STATIC_SCRATCH_BYTES bytes that is compiled into the library; every
+ * GPU that loads the library holds that array until the process exits.  It
+ * never calls cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *   Arguments as in aircache_decode_attn, without the workspace.
+ *   Limit.   2 * min(SMs, 256) * Hq * (d + 2) * 4 + 8448 bytes must fit in the array
+ *            (on a 148-SM B200: Hq * (d + 2) <= 10620, e.g. 64 heads of 128);
+ *            larger problems get AIRCACHE_ERR_STATIC_SCRATCH and nothing is enqueued.
+ *   Set-up.  The first call on each device looks up the array's device address
+ *            (with that device current).  Make that first call before any
+ *            stream capture is begun.
+ *   Sharing. All calls on a device use the one array, and the array keeps what
+ *            the last call left in it; each call therefore clears the status
+ *            word and the tickets on the stream before its kernel.  Two calls
+ *            that can overlap on the GPU (different streams without an ordering
+ *            between them) race on the array and give wrong results: order them.
+ *   Status.  The status word of the bounded waits lives inside the array and is
+ *            not visible to aircache_check_status.
+ */
+int aircache_decode_attn_static(const aircache_shape_t *shape, const aircache_ragged_t *cache, const void *q,
+                                float *out, void *cuda_stream);
 
 /*
  * Eq. 2, KV append during decoding: writes one new token's K and V

@@ -23,6 +23,7 @@ ERR_WORKSPACE_TOO_SMALL = -4
 ERR_CAPACITY = -5
 ERR_CUDA = -6
 ERR_TIMEOUT = -7
+ERR_STATIC_SCRATCH = -8
 
 
 class AirCacheError(RuntimeError):
@@ -65,6 +66,8 @@ _SIGNATURES = {
                                    C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_decode_attn": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_int64, C.c_void_p]),
+    "aircache_decode_attn_static": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p,
+                                              C.c_void_p]),
     "aircache_append": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_int32,
                                   C.c_void_p]),
     "aircache_reset_status": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
@@ -191,6 +194,14 @@ def aircache_decode_attn(sh, cache, q, out, workspace, stream=None, check=True) 
                                     _nbytes(workspace), _stream(stream))
     if check:
         _check("aircache_decode_attn", rc)
+    return rc
+
+
+def aircache_decode_attn_static(sh, cache, q, out, stream=None, check=True) -> int:
+    """aircache_decode_attn without a workspace: scratch comes from an array built into the library."""
+    rc = lib().aircache_decode_attn_static(C.byref(sh), C.byref(cache), _ptr(q), _ptr(out), _stream(stream))
+    if check:
+        _check("aircache_decode_attn_static", rc)
     return rc
 
 

@@ -114,6 +114,8 @@ const char *aircache_strerror(int code) {
         case AIRCACHE_ERR_CAPACITY: return "ragged cache capacity too small";
         case AIRCACHE_ERR_CUDA: return "CUDA error (see aircache_last_cuda_error)";
         case AIRCACHE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case AIRCACHE_ERR_STATIC_SCRATCH:
+            return "problem needs more scratch than the built-in array of aircache_decode_attn_static holds";
         default: return "unknown error code";
     }
 }
@@ -195,6 +197,16 @@ int aircache_decode_attn(const aircache_shape_t *shape, const aircache_ragged_t 
     if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return AIRCACHE_ERR_ALIGNMENT;
     if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
     return launch_decode(shape, cache, q, out, workspace, (cudaStream_t)cuda_stream);
+}
+
+int aircache_decode_attn_static(const aircache_shape_t *shape, const aircache_ragged_t *cache, const void *q,
+                                float *out, void *cuda_stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if ((rc = check_ragged(shape, cache, true))) return rc;
+    if (!q || !out) return AIRCACHE_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return AIRCACHE_ERR_ALIGNMENT;
+    return launch_decode_static(shape, cache, q, out, (cudaStream_t)cuda_stream);
 }
 
 int aircache_append(const aircache_shape_t *shape, aircache_ragged_t *cache, const void *k_new, const void *v_new,

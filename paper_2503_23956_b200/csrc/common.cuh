@@ -101,6 +101,8 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
                    cudaStream_t st);
 int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out, void *ws,
                   cudaStream_t st);
+int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out,
+                         cudaStream_t st);
 int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,
                   int32_t appended, cudaStream_t st);
 

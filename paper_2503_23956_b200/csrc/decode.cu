@@ -28,6 +28,8 @@
 // workspace, raises a CTA-wide abort flag and the kernel drains and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace aircache {
@@ -613,6 +615,57 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.tickets = ws_ptr<int32_t>(ws, w.tickets);
     p.partials = ws_ptr<float>(ws, w.partials);
     p.status = ws_ptr<uint32_t>(ws, w.status);
+    p.n_regions = s->n_layers * s->batch;
+    p.Hq = s->n_q_heads;
+    p.G = s->n_q_heads / s->n_kv_heads;
+    p.sl2 = s->scale * kLog2e;
+    return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// aircache_decode_attn_static: the same kernel with its scratch in a built-in device array
+// ---------------------------------------------------------------------------------------------
+// Status word, split-K tickets and partial slots of the decode kernel, for callers that bring no
+// workspace.  Every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[AIRCACHE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char *g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out,
+                         cudaStream_t st) {
+    int dev = 0, sms = 0;
+    AIRCACHE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return AIRCACHE_ERR_UNSUPPORTED;
+    AIRCACHE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int64_t ctas = sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas;
+    const int64_t need = kStatusBytes + 2 * ctas * s->n_q_heads * (s->head_dim + 2) * 4;
+    if (need > (int64_t)AIRCACHE_STATIC_SCRATCH_BYTES) return AIRCACHE_ERR_STATIC_SCRATCH;
+    unsigned char *base = nullptr;
+    {
+        // In host code the array's name is only a handle; its device address on the current device comes
+        // from the runtime, once per device.
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            void *ptr = nullptr;
+            AIRCACHE_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+            g_static_ptr[dev] = static_cast<unsigned char *>(ptr);
+        }
+        base = g_static_ptr[dev];
+    }
+    // The array keeps whatever the previous call left: the status word and the tickets must start at zero.
+    AIRCACHE_CUDA_TRY(cudaMemsetAsync(base, 0, kStatusBytes, st));
+    DecodeParams p;
+    p.q = (const uint16_t *)q;
+    p.out = out;
+    p.offsets = c->offsets;
+    p.lens = c->lens;
+    p.status = reinterpret_cast<uint32_t *>(base);
+    p.tickets = reinterpret_cast<int32_t *>(base + 256);
+    p.partials = reinterpret_cast<float *>(base + kStatusBytes);
     p.n_regions = s->n_layers * s->batch;
     p.Hq = s->n_q_heads;
     p.G = s->n_q_heads / s->n_kv_heads;

@@ -21,7 +21,7 @@ def declared_functions():
 
 def test_library_exports_every_declared_symbol():
     names = declared_functions()
-    assert len(names) >= 13
+    assert len(names) >= 14
     handle = C.CDLL(ac.LIB)
     for n in names:
         assert hasattr(handle, n), f"{n} declared in aircache.h but not exported"
@@ -30,8 +30,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_codes():
-    seen = {ac.aircache_strerror(c) for c in range(0, -8, -1)}
-    assert len(seen) == 8 and "unknown error code" not in seen
+    seen = {ac.aircache_strerror(c) for c in range(0, -9, -1)}
+    assert len(seen) == 9 and "unknown error code" not in seen
     assert ac.aircache_strerror(-99) == "unknown error code"
 
 
