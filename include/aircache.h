@@ -63,7 +63,7 @@ extern "C" {
 /* Problem shape, uniform over the batch. */
 typedef struct {
     int32_t n_layers;    /* L >= 1                                                                   */
-    int32_t batch;       /* B >= 1; L * B <= 2048                                                    */
+    int32_t batch;       /* B >= 1; L * B <= 1920                                                    */
     int32_t n_q_heads;   /* Hq, a multiple of n_kv_heads with Hq / Hkv <= 16                         */
     int32_t n_kv_heads;  /* Hkv in {1, 2, 4, 8}                                                      */
     int32_t head_dim;    /* d in {64, 128}                                                           */
@@ -204,7 +204,7 @@ int aircache_decode_attn(const aircache_shape_t *shape, const aircache_ragged_t 
  * never calls cudaMalloc, cudaFree or any other allocating routine.
  *
  *   Arguments as in aircache_decode_attn, without the workspace.
- *   Limit.   2 * min(SMs, 256) * Hq * (d + 2) * 4 + 8448 bytes must fit in the array
+ *   Limit.   2 * min(SMs, 256) * Hq * (d + 2) * 4 + 7936 bytes must fit in the array
  *            (on a 148-SM B200: Hq * (d + 2) <= 10620, e.g. 64 heads of 128);
  *            larger problems get AIRCACHE_ERR_STATIC_SCRATCH and nothing is enqueued.
  *   Set-up.  The first call on each device looks up the array's device address

@@ -37,6 +37,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static", "--threads", "0"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("AIRCACHE_NVCC_FLAGS", "").split()
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -72,7 +72,7 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.alloc_share = take(LB * 8);
     w.alloc_active = take(LB * 4);
     w.kept = take(LB * s->n_visual * 4);
-    w.partials = take((int64_t)2 * kMaxDecodeCtas * s->n_q_heads * (s->head_dim + 2) * 4);
+    w.partials = take((int64_t)2 * kMaxDecodeCtas * partial_slot_floats(s->n_q_heads, s->head_dim) * 4);
     w.total = off;
     return w;
 }

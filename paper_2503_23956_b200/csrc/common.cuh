@@ -11,7 +11,7 @@ namespace aircache {
 
 constexpr int kMaxWindow = 64;
 constexpr int kMaxGroup = 16;         // query heads per KV head
-constexpr int kMaxRegions = 2048;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
+constexpr int kMaxRegions = 1920;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
 constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;
@@ -48,6 +48,12 @@ int check_full(const aircache_shape_t *s, const aircache_full_t *f);
 int64_t kept_per_sequence(const aircache_shape_t *s, double ratio);
 
 inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Floats of one split-K partial slot of the decode kernel: [Hq, d] accumulator, Hq maxima, Hq sums, padded so
+// that every slot starts on a 16-byte boundary.
+__host__ __device__ inline int64_t partial_slot_floats(int n_q_heads, int head_dim) {
+    return ((int64_t)n_q_heads * (head_dim + 2) + 3) / 4 * 4;
+}
 
 // Elite rows one KV group can have at most, padded to the MMA tile of 8 rows.
 inline int score_row_cap(const aircache_shape_t *s) {

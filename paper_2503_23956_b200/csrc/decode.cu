@@ -4,7 +4,9 @@
 // Work decomposition.  A "unit" is CH consecutive rows of one region (all KV heads, K and V).  Region r
 // has ceil(lens[r] / CH) units; every CTA first scans these counts into a prefix P (shared memory), then
 // takes the contiguous unit range [c * upc, (c+1) * upc) of the global unit list, upc = ceil(total / CTAs).
-// The load is therefore balanced to one unit regardless of how ragged the regions are.  Consecutive units
+// The load is therefore balanced to one unit regardless of how ragged the regions are.  When there are
+// few regions and cutting each one into pieces of at most upc units needs no more CTAs than the grid has,
+// the pieces are aligned to regions instead (same longest piece, but one query load and one flush per CTA).  Consecutive units
 // of one region accumulate in registers; a region that lies wholly inside one CTA's range is finished and
 // written by that CTA, otherwise the CTA writes an unnormalised partial (running max, sum, accumulator) and
 // takes a ticket of the region; the CTA that draws the last ticket merges the region's partials in CTA
@@ -37,6 +39,21 @@ namespace aircache {
 namespace {
 
 constexpr uint32_t kSpinLimit = 1u << 22;
+
+// Development aid, compiled out unless AIRCACHE_DECODE_TRACE is defined: thread 0 of every CTA stores
+// %globaltimer at a few points of the kernel into the unused tail of the partial slots.
+#ifdef AIRCACHE_DECODE_TRACE
+#define DECODE_TRACE(idx)                                                                                   \
+    do {                                                                                                    \
+        if (threadIdx.x == 0) {                                                                             \
+            unsigned long long _t;                                                                          \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));                                          \
+            reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 16 + (idx)] = _t; \
+        }                                                                                                   \
+    } while (0)
+#else
+#define DECODE_TRACE(idx) do { } while (0)
+#endif
 
 struct DecodeParams {
     const uint16_t *q;       // [L*B, Hq, D]
@@ -91,6 +108,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
+// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier (16-byte aligned, size % 16 == 0).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+                 : "memory");
+}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -125,14 +148,30 @@ struct DecodeCfg {
     // merge buffer: one slot per consumer warp with ks > 0
     static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 2));
     static constexpr int MERGE_BYTES = HKV * (KSPLIT - 1) * MERGE_FLOATS_PER_WARP * 4;
-    static constexpr int PLAN_BYTES = (kMaxRegions + 2) * 4;
-    // ring depth: what fits beside the merge buffer and the plan in the 227 KB a CTA may use (3 KB are
-    // left for static shared memory and the 1 KB alignment slack), at most 4 stages
-    static constexpr int FIT = (232448 - 3072 - 1024 - MERGE_BYTES - PLAN_BYTES - 256) / STAGE_BYTES;
+    // the prologue's scan scratch lives in the same bytes as the merge buffer (used before the first flush)
+    static constexpr int SCAN_BYTES = THREADS * 4;
+    static constexpr int MERGE_STAGE_BYTES = 16384;            // weights [partials][Hq] of the final merge
+    static constexpr int SCRATCH_MIN = SCAN_BYTES > MERGE_STAGE_BYTES ? SCAN_BYTES : MERGE_STAGE_BYTES;
+    static constexpr int SCRATCH_BYTES = ((MERGE_BYTES > SCRATCH_MIN ? MERGE_BYTES : SCRATCH_MIN) + 15) / 16 * 16;
+    static constexpr int PLAN_BYTES = (kMaxRegions + 2) * 4;   // unit prefix
+    static constexpr int OFFS_BYTES = kMaxRegions * 4;         // first row of every region
+    // ring depth: what fits beside the scratch and the tables in the 227 KB a CTA may use (1.5 KB are left
+    // for static shared memory, 1 KB for the alignment slack), at most 4 stages
+    static constexpr int FIT = (232448 - 1536 - 1024 - SCRATCH_BYTES - PLAN_BYTES - OFFS_BYTES - 256) / STAGE_BYTES;
     static constexpr int NSTAGE = FIT > 4 ? 4 : FIT;
     static_assert(NSTAGE >= 2, "decode pipeline needs two stages");
-    static constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + MERGE_BYTES + PLAN_BYTES + 256;
+    static constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + SCRATCH_BYTES + PLAN_BYTES + OFFS_BYTES + 256;
 };
+
+// a / b for a >= 0, b > 0, through the fp32 divider when both are below 2^23 (an integer division by a run-time
+// divisor costs several hundred cycles of the prologue otherwise)
+__device__ __forceinline__ int small_div(int a, int b) {
+    if (a >= (1 << 23) || b >= (1 << 23)) return a / b;
+    int q = (int)__fdividef((float)a, (float)b);
+    if (q * b > a) --q;
+    if ((q + 1) * b <= a) ++q;
+    return q;
+}
 
 // largest r with P[r] <= u (P non-decreasing, P[0] = 0, u < P[n])
 __device__ __forceinline__ int find_region(const int *P, int n, int u) {
@@ -150,28 +189,42 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     using C = DecodeCfg<D, HKV, G_HI>;
     constexpr int KSPLIT = C::KSPLIT, CH = C::CH, NCW = C::NCW, NROW = C::NROW, kStages = C::NSTAGE;
 
+    DECODE_TRACE(0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *s_stage = smem;
     float *s_merge = reinterpret_cast<float *>(smem + kStages * C::STAGE_BYTES);
-    int *s_P = reinterpret_cast<int *>(smem + kStages * C::STAGE_BYTES + C::MERGE_BYTES);
-    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + kStages * C::STAGE_BYTES + C::MERGE_BYTES + C::PLAN_BYTES);
-    __shared__ int s_part[C::THREADS];
+    int *s_part = reinterpret_cast<int *>(s_merge);   // scan scratch of the prologue, same bytes
+    int *s_P = reinterpret_cast<int *>(smem + kStages * C::STAGE_BYTES + C::SCRATCH_BYTES);
+    int *s_off = reinterpret_cast<int *>(smem + kStages * C::STAGE_BYTES + C::SCRATCH_BYTES + C::PLAN_BYTES);
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + kStages * C::STAGE_BYTES + C::SCRATCH_BYTES + C::PLAN_BYTES +
+                                                   C::OFFS_BYTES);
+    __shared__ int s_Q[kMaxDecodeCtas + 1];   // region-aligned mode: first CTA of every region
     __shared__ int s_abort;
     __shared__ int s_last;
+    __shared__ int s_aligned;
 
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int n = p.n_regions;
+    const int n_ctas = (int)gridDim.x;
+    if (wid == NCW && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+    }
 
-    // ---- unit prefix of all regions (every CTA computes the same table) ----
+    // ---- unit prefix and first row of all regions (every CTA computes the same tables) ----
     {
         const int per = (n + C::THREADS - 1) / C::THREADS;
         const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
         int local = 0;
-        for (int i = i0; i < i1; ++i) local += (max(p.lens[i], 0) + CH - 1) / CH;
+        for (int i = i0; i < i1; ++i) {
+            local += (max(p.lens[i], 0) + CH - 1) / CH;
+            s_off[i] = (int)p.offsets[i];
+        }
         s_part[tid] = local;
         if (tid == 0) s_abort = 0;
         __syncthreads();
+        DECODE_TRACE(12);
         if (wid == 0) {
             // warp 0 turns s_part into an exclusive prefix
             constexpr int PER_LANE = (C::THREADS + 31) / 32;
@@ -205,37 +258,84 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 mbar_init(smem_u32(&s_bar[s]), 1);             // full: the producer's expect_tx arrival
                 mbar_init(smem_u32(&s_bar[kStages + s]), NCW);  // empty: one arrival per consumer warp
             }
+            mbar_init(smem_u32(&s_bar[2 * kStages]), 1);        // partials staged for the final merge
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncthreads();
     }
+    DECODE_TRACE(13);
     const int total = s_P[n];
+    const int upc = max(1, small_div(total + n_ctas - 1, n_ctas));
+
+    // ---- schedule.  Balanced mode: CTA c takes units [c * upc, (c+1) * upc) of the global list.
+    // Region-aligned mode (few regions, each cut into pieces of at most upc units, if that needs no more
+    // CTAs than there are): every CTA works on one region only, so it reloads no query and flushes once.
+    if (wid == 0) {
+        // pieces per region and their exclusive prefix, 32 regions per round (rolled: this runs once)
+        const bool few = n <= n_ctas;
+        int carry = 0;
+#pragma unroll 1
+        for (int base = 0; few && base <= n; base += 32) {
+            const int r = base + lane;
+            const int v = r < n ? small_div(s_P[r + 1] - s_P[r] + upc - 1, upc) : 0;
+            int incl = v;
+#pragma unroll
+            for (int sh = 1; sh < 32; sh <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+                if (lane >= sh) incl += o;
+            }
+            if (r <= n) s_Q[r] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) s_aligned = (few && total > 0 && carry <= n_ctas) ? 1 : 0;
+    }
+    __syncthreads();
+    DECODE_TRACE(14);
+    const bool aligned = s_aligned != 0;
+
     // a region without rows yields zeros
-    for (int r = blockIdx.x; r < n; r += gridDim.x) {
+    for (int r = blockIdx.x; r < n; r += n_ctas) {
         if (s_P[r + 1] == s_P[r])
             for (int i = tid; i < p.Hq * D; i += C::THREADS) p.out[(int64_t)r * p.Hq * D + i] = 0.f;
     }
-    const int upc = max(1, (total + (int)gridDim.x - 1) / (int)gridDim.x);
-    const int u0 = min(total, (int)blockIdx.x * upc), u1 = min(total, u0 + upc);
+    int u0, u1;
+    if (aligned) {
+        const int c = (int)blockIdx.x;
+        if (c >= s_Q[n]) return;
+        const int r = find_region(s_Q, n, c);      // largest r with s_Q[r] <= c: the region this CTA cuts
+        const int pieces = s_Q[r + 1] - s_Q[r], j = c - s_Q[r], units = s_P[r + 1] - s_P[r];
+        u0 = s_P[r] + small_div(units * j, pieces);          // units * pieces < 2^24: both are at most a few thousand
+        u1 = s_P[r] + small_div(units * (j + 1), pieces);
+    } else {
+        u0 = min(total, (int)blockIdx.x * upc);
+        u1 = min(total, u0 + upc);
+    }
     if (u0 >= u1) return;
+    DECODE_TRACE(1);
+    // CTAs that hold a piece of region r, and the partial slot CTA c uses for it
+    auto span_of = [&](int r, int &c0, int &c1) {
+        if (aligned) { c0 = s_Q[r]; c1 = s_Q[r + 1] - 1; }
+        else { c0 = s_P[r] / upc; c1 = (s_P[r + 1] - 1) / upc; }
+    };
+    auto slot_of = [&](int c, int r) { return aligned ? 2 * c : 2 * c + ((s_P[r] <= c * upc) ? 0 : 1); };
 
     if (wid == NCW) {
         // =============================== producer warp ===============================
         if (lane == 0) {
             int r = find_region(s_P, n, u0);
-            int64_t row_base = p.offsets[r];
+            int row_base = s_off[r];
             int it = 0;
             bool ok = true;
             for (int u = u0; u < u1 && ok; ++u, ++it) {
                 if (u >= s_P[r + 1]) {
                     while (u >= s_P[r + 1]) ++r;
-                    row_base = p.offsets[r];
+                    row_base = s_off[r];
                 }
                 const int s = it % kStages;
                 if (it >= kStages)
                     ok = mbar_wait(smem_u32(&s_bar[kStages + s]), ((it / kStages) & 1) ^ 1, &s_abort, p.status, 1);
                 if (!ok) break;
-                const int row0 = (int)(row_base + (int64_t)(u - s_P[r]) * CH);
+                const int row0 = row_base + (u - s_P[r]) * CH;
                 const uint32_t full = smem_u32(&s_bar[s]);
                 mbar_expect_tx(full, C::STAGE_BYTES);
                 const uint32_t dst = smem_u32(s_stage + s * C::STAGE_BYTES);
@@ -265,6 +365,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int gid = lane >> 2, t = lane & 3;
     const int G = p.G;
 
+    int n_flush = 0;  // flushes done so far (trace slots only)
     uint32_t qa[D / 16][4];
     float oacc[D / 8][4];
     float m_run[2], l_run[2];
@@ -348,8 +449,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) =
                             make_float2(oacc[nd][2 * i] * inv, oacc[nd][2 * i + 1] * inv);
                 } else {
-                    const int slot = 2 * (int)blockIdx.x + ((s_P[r] <= u0) ? 0 : 1);
-                    float *base = p.partials + (size_t)slot * p.Hq * (D + 2);
+                    const int slot = slot_of((int)blockIdx.x, r);
+                    float *base = p.partials + (size_t)slot * partial_slot_floats(p.Hq, D);
                     float *o = base + (size_t)h * D;
 #pragma unroll
                     for (int nd = 0; nd < D / 8; ++nd)
@@ -367,55 +468,108 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // the region's last ticket merges all partials in CTA order
             __threadfence();
             consumer_bar(NCW * 32);
-            const int c0 = s_P[r] / upc, c1 = (s_P[r + 1] - 1) / upc;
+            int c0, c1;
+            span_of(r, c0, c1);
             if (tid == 0) {
                 const int tk = atomicAdd(p.tickets + r, 1);
                 s_last = (tk == c1 - c0);
-                if (s_last) p.tickets[r] = 0;
-                __threadfence();
+                if (s_last) __threadfence();
             }
             consumer_bar(NCW * 32);
+            DECODE_TRACE(4 + 3 * n_flush);
             if (s_last) {
-                const size_t slot_floats = (size_t)p.Hq * (D + 2);
-                const int P0 = s_P[r];
-                // every thread owns float4 columns of the [Hq, D] result; the partials are visited eight at a
-                // time with all their loads in flight together, merged online in CTA order
-                for (int i = tid; i < p.Hq * D / 4; i += NCW * 32) {
-                    const int h = (i * 4) / D;
-                    float M = -INFINITY, den = 0.f;
-                    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int cb = c0; cb <= c1; cb += 8) {
-                        float mm[8], ll[8];
-                        float4 aa[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int c = min(cb + j, c1);
-                            const int slot = 2 * c + ((P0 <= c * upc) ? 0 : 1);
-                            const float *base = p.partials + slot * slot_floats;
-                            mm[j] = __ldcg(base + (size_t)p.Hq * D + h);
-                            ll[j] = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
-                            aa[j] = __ldcg(reinterpret_cast<const float4 *>(base) + i);
-                        }
-                        float mx = -INFINITY;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (cb + j > c1) mm[j] = -INFINITY;
-                            mx = fmaxf(mx, mm[j]);
-                        }
-                        const float Mn = fmaxf(M, mx);
-                        const float sc = exp2_or_zero(M, Mn);
-                        num.x *= sc; num.y *= sc; num.z *= sc; num.w *= sc; den *= sc;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float w = exp2_or_zero(mm[j], Mn);
-                            num.x += aa[j].x * w; num.y += aa[j].y * w; num.z += aa[j].z * w; num.w += aa[j].w * w;
-                            den += ll[j] * w;
-                        }
-                        M = Mn;
+                if (tid == 0) p.tickets[r] = 0;   // ready for the next call
+                const size_t slot_floats = (size_t)partial_slot_floats(p.Hq, D);
+                const int items = p.Hq * D / 4;
+                const int np = c1 - c0 + 1;
+                float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)r * p.Hq * D);
+                if (uend == u1 && (size_t)np * slot_floats * 4 <= (size_t)kStages * C::STAGE_BYTES) {
+                    // This CTA has no unit left, so the ring is empty: pull all partials of the region into it
+                    // with bulk copies (one round trip for everything), then merge out of shared memory.  The
+                    // loops below are rolled on purpose: the code runs once and cold instructions cost more
+                    // than the arithmetic.
+                    const uint32_t bar = smem_u32(&s_bar[2 * kStages]);
+                    const uint32_t slot_bytes = (uint32_t)(slot_floats * 4);
+                    if (tid == 0) {
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                        mbar_expect_tx(bar, np * slot_bytes);
+#pragma unroll 1
+                        for (int c = 0; c < np; ++c)
+                            bulk_load(smem_u32(s_stage) + c * slot_bytes, p.partials + slot_of(c0 + c, r) * slot_floats,
+                                      slot_bytes, bar);
                     }
-                    const float inv = den > 0.f ? 1.0f / den : 0.f;
-                    reinterpret_cast<float4 *>(p.out + (int64_t)r * p.Hq * D)[i] =
-                        make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+                    if (mbar_wait(bar, 0, &s_abort, p.status, 3)) {
+                        DECODE_TRACE(9);
+                        const float *sp = reinterpret_cast<const float *>(s_stage);
+                        float *wgt = s_merge;   // [np][Hq] weights exp2(m_c - M) / sum
+#pragma unroll 1
+                        for (int h = tid; h < p.Hq; h += NCW * 32) {
+                            float M = -INFINITY, den = 0.f;
+#pragma unroll 1
+                            for (int c = 0; c < np; ++c) M = fmaxf(M, sp[c * slot_floats + p.Hq * D + h]);
+#pragma unroll 1
+                            for (int c = 0; c < np; ++c)
+                                den += sp[c * slot_floats + p.Hq * (D + 1) + h] *
+                                       exp2_or_zero(sp[c * slot_floats + p.Hq * D + h], M);
+                            const float inv = den > 0.f ? 1.0f / den : 0.f;
+#pragma unroll 1
+                            for (int c = 0; c < np; ++c)
+                                wgt[c * p.Hq + h] = exp2_or_zero(sp[c * slot_floats + p.Hq * D + h], M) * inv;
+                        }
+                        consumer_bar(NCW * 32);
+                        DECODE_TRACE(10);
+#pragma unroll 1
+                        for (int i = tid; i < items; i += NCW * 32) {
+                            const int h = (i * 4) / D;
+                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+                            for (int c = 0; c < np; ++c) {
+                                const float4 a = reinterpret_cast<const float4 *>(sp + c * slot_floats)[i];
+                                const float w = wgt[c * p.Hq + h];
+                                acc.x += a.x * w; acc.y += a.y * w; acc.z += a.z * w; acc.w += a.w * w;
+                            }
+                            o4[i] = acc;
+                        }
+                    }
+                } else {
+                    // Mid-stream (the ring is busy) or too many partials for it: online merge straight from
+                    // global memory, eight partials' loads in flight per column.
+#pragma unroll 1
+                    for (int i = tid; i < items; i += NCW * 32) {
+                        const int h = (i * 4) / D;
+                        float M = -INFINITY, den = 0.f;
+                        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+                        for (int cb = c0; cb <= c1; cb += 8) {
+                            float mm[8], ll[8];
+                            float4 aa[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float *base = p.partials + slot_of(min(cb + j, c1), r) * slot_floats;
+                                mm[j] = __ldcg(base + (size_t)p.Hq * D + h);
+                                ll[j] = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
+                                aa[j] = __ldcg(reinterpret_cast<const float4 *>(base) + i);
+                            }
+                            float mx = -INFINITY;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (cb + j > c1) mm[j] = -INFINITY;
+                                mx = fmaxf(mx, mm[j]);
+                            }
+                            const float Mn = fmaxf(M, mx);
+                            const float sc = exp2_or_zero(M, Mn);
+                            num.x *= sc; num.y *= sc; num.z *= sc; num.w *= sc; den *= sc;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float w = exp2_or_zero(mm[j], Mn);
+                                num.x += aa[j].x * w; num.y += aa[j].y * w; num.z += aa[j].z * w; num.w += aa[j].w * w;
+                                den += ll[j] * w;
+                            }
+                            M = Mn;
+                        }
+                        const float inv = den > 0.f ? 1.0f / den : 0.f;
+                        o4[i] = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+                    }
                 }
             }
         }
@@ -429,7 +583,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     bool ok = true;
     for (int u = u0; u < u1; ++u, ++it) {
         if (u >= s_P[r + 1]) {
+            DECODE_TRACE(3 + 3 * n_flush);
             flush(r, seg_start, u);
+            DECODE_TRACE(5 + 3 * n_flush);
+            n_flush = n_flush < 2 ? n_flush + 1 : 2;
             while (u >= s_P[r + 1]) ++r;
             seg_start = u;
             len = p.lens[r];
@@ -438,6 +595,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int s = it % kStages;
         ok = mbar_wait(smem_u32(&s_bar[s]), (it / kStages) & 1, &s_abort, p.status, 2);
         if (!ok) break;
+        if (it == 0) DECODE_TRACE(2);
         const int j0 = (u - s_P[r]) * CH + ks * 16;  // first row of this warp's block inside the region
         if (j0 < len) {
             const uint32_t k_base = smem_u32(s_stage + s * C::STAGE_BYTES) + g * C::HALVES * C::SUBTILE;
@@ -525,7 +683,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_bar[kStages + s]));
     }
+    DECODE_TRACE(3 + 3 * n_flush);
     if (ok) flush(r, seg_start, u1);
+    DECODE_TRACE(5 + 3 * n_flush);
+    DECODE_TRACE(15);
+    (void)n_flush;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -642,7 +804,7 @@ int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, 
     if (dev < 0 || dev >= kMaxDevices) return AIRCACHE_ERR_UNSUPPORTED;
     AIRCACHE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int64_t ctas = sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas;
-    const int64_t need = kStatusBytes + 2 * ctas * s->n_q_heads * (s->head_dim + 2) * 4;
+    const int64_t need = kStatusBytes + 2 * ctas * partial_slot_floats(s->n_q_heads, s->head_dim) * 4;
     if (need > (int64_t)AIRCACHE_STATIC_SCRATCH_BYTES) return AIRCACHE_ERR_STATIC_SCRATCH;
     unsigned char *base = nullptr;
     {

@@ -29,6 +29,8 @@ CASES = {
     "g16": small("g16", L=2, Hq=16, Hkv=1, d=64, B=2, Nv=257, Nt=17, W=5),   # 16 query heads per KV head
     "kv2": small("kv2", L=2, Hq=12, Hkv=2, d=128, B=2, Nv=515, Nt=64, W=64),  # widest window
     "kv1": small("kv1", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=130, Nt=9, W=9),
+    # long regions cut across many CTAs with an odd head count (padded partial slots, multi-round merge)
+    "kv1long": small("kv1long", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=9000, Nt=9, W=4, ratio=0.9),
 }
 
 
