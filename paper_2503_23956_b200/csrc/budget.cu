@@ -1,11 +1,13 @@
 // aircache_budget: strength and skewness of every region's importance distribution (Eq. 9-10), the
 // layer-wise budget of Eq. 11 turned into integer row counts, and the row offsets of the ragged cache.
 //
-//   moments_kernel   one CTA per region: three fp64 block reductions (sum; squared deviations; cubed
-//                    standardised deviations) over the fp32 scores, fixed reduction tree.
-//   allocate_kernel  one CTA: thread b walks the layers of sequence b in order and performs the capped
-//                    proportional split with largest-remainder rounding in fp64, every operation
-//                    individually rounded (no fused multiply-add), then all threads scan the region sizes.
+// One launch.  Every CTA reduces one region (three fp64 block reductions over the fp32 scores, which it
+// keeps in registers: sum; squared deviations; cubed standardised deviations; fixed reduction tree).  The
+// CTA that finishes last (a ticket in the workspace, put back to zero for the next call) then runs the
+// allocation for all sequences: one warp per sequence, sums over the layers taken by one lane in layer
+// order and every fp64 operation individually rounded (no fused multiply-add), so that the integer
+// budgets are the ones the sequential definition gives; divisions, floors and the ranking of the
+// fractional parts run across the lanes.  Finally the same CTA scans the region sizes into offsets.
 #include <math.h>
 
 #include "common.cuh"
@@ -14,7 +16,19 @@ namespace aircache {
 
 namespace {
 
-constexpr int kMomThreads = 256;
+constexpr int kThreads = 512;
+constexpr int kPerThread = 16;   // scores a thread keeps in registers (covers N_v <= 8192; beyond, re-read)
+
+struct BudgetParams {
+    const float *scores;     // [L*B, Nv]
+    double *strength, *skewness;  // [L,B]
+    int32_t *budgets;        // [L,B]
+    int64_t *offsets;        // [L*B+1]
+    int32_t *lens;           // [L*B]
+    uint32_t *ticket;        // zero between calls
+    int L, B, Nv, Nt, slack, mode;
+    long long total_kept;    // T per sequence
+};
 
 __device__ __forceinline__ double block_sum(double v, double *s_part) {
 #pragma unroll
@@ -24,143 +38,199 @@ __device__ __forceinline__ double block_sum(double v, double *s_part) {
     if (lane == 0) s_part[warp] = v;
     __syncthreads();
     double tot = 0.0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot = __dadd_rn(tot, s_part[w]);
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) tot = __dadd_rn(tot, s_part[w]);
     return tot;
 }
 
-// Eq. 9 and Eq. 10 (adjusted Fisher-Pearson coefficient, sample standard deviation).
-__global__ void __launch_bounds__(kMomThreads) moments_kernel(const float *__restrict__ scores, int n_visual,
-                                                              double *__restrict__ strength,
-                                                              double *__restrict__ skewness) {
-    __shared__ double s_part[kMomThreads / 32];
-    const float *x = scores + (int64_t)blockIdx.x * n_visual;
-    const double n = (double)n_visual;
-
-    double s = 0.0;
-    for (int i = threadIdx.x; i < n_visual; i += kMomThreads) s = __dadd_rn(s, (double)x[i]);
-    s = block_sum(s, s_part);
-    const double mu = __ddiv_rn(s, n);
-
-    double ss = 0.0;
-    for (int i = threadIdx.x; i < n_visual; i += kMomThreads) {
-        const double c = __dsub_rn((double)x[i], mu);
-        ss = __dadd_rn(ss, __dmul_rn(c, c));
-    }
-    ss = block_sum(ss, s_part);
-    const double sigma = __dsqrt_rn(__ddiv_rn(ss, __dsub_rn(n, 1.0)));
-
-    double cube = 0.0;
-    if (sigma > 0.0) {
-        for (int i = threadIdx.x; i < n_visual; i += kMomThreads) {
-            const double zc = __ddiv_rn(__dsub_rn((double)x[i], mu), sigma);
-            cube = __dadd_rn(cube, __dmul_rn(__dmul_rn(zc, zc), zc));
-        }
-    }
-    cube = block_sum(cube, s_part);
-    if (threadIdx.x == 0) {
-        strength[blockIdx.x] = s;
-        const double pre = __ddiv_rn(n, __dmul_rn(__dsub_rn(n, 1.0), __dsub_rn(n, 2.0)));
-        skewness[blockIdx.x] = (sigma > 0.0) ? __dmul_rn(pre, cube) : 0.0;
-    }
+__device__ __forceinline__ double warp_bcast(double v, int src) {
+    return __shfl_sync(0xffffffffu, v, src);
 }
 
-struct AllocParams {
-    const double *strength, *skewness;  // [L,B]
-    double *w, *share;                  // [L,B] scratch
-    int32_t *active;                    // [L,B] scratch
-    int32_t *budgets;                   // [L,B]
-    int64_t *offsets;                   // [L*B+1]
-    int32_t *lens;                      // [L*B]
-    int L, B, Nv, Nt, slack, mode;
-    long long total_kept;               // T per sequence
-};
-
-constexpr int kAllocThreads = 1024;
-
-__global__ void __launch_bounds__(kAllocThreads) allocate_kernel(AllocParams p) {
-    const int L = p.L, B = p.B;
-    // ---- Eq. 11 + integer budgets, one thread per sequence ----
-    for (int b = threadIdx.x; b < B; b += kAllocThreads) {
-        double mean_t = 0.0, mean_k = 0.0;
+// Eq. 11 and the integer budgets of sequence b, by one warp.  st/sk/w/share are [L*B] arrays in shared
+// memory, element (l, b) at l*B + b; act flags layers that still take part in the proportional split.
+__device__ void allocate_sequence(const BudgetParams &p, int b, const double *st, const double *sk, double *w,
+                                  double *share, unsigned char *act, int *bud) {
+    const int L = p.L, B = p.B, lane = threadIdx.x & 31;
+    // across-layer means: one lane, layer order (this fixes the rounding of the sums)
+    double mean_t = 0.0, mean_k = 0.0;
+    if (lane == 0) {
         for (int l = 0; l < L; ++l) {
-            mean_t = __dadd_rn(mean_t, p.strength[l * B + b]);
-            const double sk = p.skewness[l * B + b];
-            mean_k = __dadd_rn(mean_k, sk > 0.0 ? sk : 0.0);
+            mean_t = __dadd_rn(mean_t, st[l * B + b]);
+            const double s = sk[l * B + b];
+            mean_k = __dadd_rn(mean_k, s > 0.0 ? s : 0.0);
         }
         mean_t = __ddiv_rn(mean_t, (double)L);
         mean_k = __ddiv_rn(mean_k, (double)L);
-        for (int l = 0; l < L; ++l) {
-            const double st = p.strength[l * B + b];
-            double sk = p.skewness[l * B + b];
-            if (sk < 0.0) sk = 0.0;
-            const double nt = mean_t > 0.0 ? __ddiv_rn(st, mean_t) : 1.0;
-            const double nk = mean_k > 0.0 ? __ddiv_rn(sk, mean_k) : 1.0;
-            double w;
-            if (p.mode == 0) w = __dmul_rn(0.5, __dadd_rn(nt, nk));
-            else if (p.mode == 1) w = nt;
-            else if (p.mode == 2) w = nk;
-            else w = 1.0;
-            p.w[l * B + b] = w;
-            p.active[l * B + b] = 1;
-        }
-        long long R = p.total_kept;
-        // capped proportional split: a layer whose share reaches Nv keeps everything, the rest re-share
-        for (;;) {
-            double wsum = 0.0;
-            int n_active = 0;
+    }
+    mean_t = warp_bcast(mean_t, 0);
+    mean_k = warp_bcast(mean_k, 0);
+    for (int l = lane; l < L; l += 32) {
+        const double t = st[l * B + b];
+        double s = sk[l * B + b];
+        if (s < 0.0) s = 0.0;
+        const double nt = mean_t > 0.0 ? __ddiv_rn(t, mean_t) : 1.0;
+        const double nk = mean_k > 0.0 ? __ddiv_rn(s, mean_k) : 1.0;
+        double ww;
+        if (p.mode == 0) ww = __dmul_rn(0.5, __dadd_rn(nt, nk));
+        else if (p.mode == 1) ww = nt;
+        else if (p.mode == 2) ww = nk;
+        else ww = 1.0;
+        w[l * B + b] = ww;
+        act[l * B + b] = 1;
+    }
+    __syncwarp();
+    long long R = p.total_kept;
+    // capped proportional split: a layer whose share reaches Nv keeps everything, the rest re-share
+    for (;;) {
+        double wsum = 0.0;
+        int n_active = 0;
+        if (lane == 0) {
             for (int l = 0; l < L; ++l)
-                if (p.active[l * B + b]) { wsum = __dadd_rn(wsum, p.w[l * B + b]); ++n_active; }
-            if (n_active == 0) break;
-            for (int l = 0; l < L; ++l) {
-                if (!p.active[l * B + b]) continue;
-                p.share[l * B + b] = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, p.w[l * B + b]), wsum)
-                                                : __ddiv_rn((double)R, (double)n_active);
+                if (act[l * B + b]) { wsum = __dadd_rn(wsum, w[l * B + b]); ++n_active; }
+        }
+        wsum = warp_bcast(wsum, 0);
+        n_active = __shfl_sync(0xffffffffu, n_active, 0);
+        if (n_active == 0) break;
+        int moved = 0;
+        for (int l = lane; l < L; l += 32) {
+            if (!act[l * B + b]) continue;
+            const double sh = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, w[l * B + b]), wsum)
+                                         : __ddiv_rn((double)R, (double)n_active);
+            share[l * B + b] = sh;
+            if (sh >= (double)p.Nv) {
+                bud[l * B + b] = p.Nv;
+                act[l * B + b] = 0;
+                ++moved;
             }
-            bool moved = false;
-            for (int l = 0; l < L; ++l) {
-                if (p.active[l * B + b] && p.share[l * B + b] >= (double)p.Nv) {
-                    p.budgets[l * B + b] = p.Nv;
-                    p.active[l * B + b] = 0;
-                    R -= p.Nv;
-                    moved = true;
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) moved += __shfl_xor_sync(0xffffffffu, moved, s);
+        __syncwarp();
+        if (moved == 0) break;
+        R -= (long long)moved * p.Nv;
+    }
+    // floors, then the largest fractional parts (ties to the lower layer) take one more row each
+    int given = 0;
+    for (int l = lane; l < L; l += 32) {
+        if (!act[l * B + b]) continue;
+        const double sh = share[l * B + b];
+        const int f = (int)floor(sh);
+        bud[l * B + b] = f;
+        given += f;
+        share[l * B + b] = __dsub_rn(sh, (double)f);
+    }
+    long long given_all = given;
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) given_all += __shfl_xor_sync(0xffffffffu, given_all, s);
+    __syncwarp();
+    const long long left = R - given_all;
+    // a layer gets the extra row iff fewer than `left` active layers precede it in the order
+    // (fraction descending, layer ascending): the same set the one-at-a-time selection picks
+    for (int l = lane; l < L; l += 32) {
+        if (!act[l * B + b]) continue;
+        const double fr = share[l * B + b];
+        long long rank = 0;
+        for (int l2 = 0; l2 < L; ++l2) {
+            if (!act[l2 * B + b]) continue;
+            const double f2 = share[l2 * B + b];
+            rank += (f2 > fr) || (f2 == fr && l2 < l);
+        }
+        if (rank < left) bud[l * B + b] += 1;
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    __shared__ double s_part[kThreads / 32];
+    __shared__ int s_is_last;
+    const int tid = threadIdx.x;
+    const int LB = p.L * p.B;
+
+    // ---------------- Eq. 9 and Eq. 10 of region blockIdx.x ----------------
+    {
+        const float *x = p.scores + (int64_t)blockIdx.x * p.Nv;
+        const double n = (double)p.Nv;
+        float v[kPerThread];
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k) {
+            const int i = tid + k * kThreads;
+            v[k] = i < p.Nv ? x[i] : 0.f;
+        }
+        const bool spill = p.Nv > kThreads * kPerThread;
+        double s = 0.0;
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k)
+            if (tid + k * kThreads < p.Nv) s = __dadd_rn(s, (double)v[k]);
+        if (spill)
+            for (int i = tid + kPerThread * kThreads; i < p.Nv; i += kThreads) s = __dadd_rn(s, (double)x[i]);
+        s = block_sum(s, s_part);
+        const double mu = __ddiv_rn(s, n);
+
+        double ss = 0.0;
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k)
+            if (tid + k * kThreads < p.Nv) { const double c = __dsub_rn((double)v[k], mu); ss = __dadd_rn(ss, __dmul_rn(c, c)); }
+        if (spill)
+            for (int i = tid + kPerThread * kThreads; i < p.Nv; i += kThreads) {
+                const double c = __dsub_rn((double)x[i], mu);
+                ss = __dadd_rn(ss, __dmul_rn(c, c));
+            }
+        ss = block_sum(ss, s_part);
+        const double sigma = __dsqrt_rn(__ddiv_rn(ss, __dsub_rn(n, 1.0)));
+
+        double cube = 0.0;
+        if (sigma > 0.0) {
+#pragma unroll
+            for (int k = 0; k < kPerThread; ++k)
+                if (tid + k * kThreads < p.Nv) {
+                    const double zc = __ddiv_rn(__dsub_rn((double)v[k], mu), sigma);
+                    cube = __dadd_rn(cube, __dmul_rn(__dmul_rn(zc, zc), zc));
                 }
-            }
-            if (!moved) break;
+            if (spill)
+                for (int i = tid + kPerThread * kThreads; i < p.Nv; i += kThreads) {
+                    const double zc = __ddiv_rn(__dsub_rn((double)x[i], mu), sigma);
+                    cube = __dadd_rn(cube, __dmul_rn(__dmul_rn(zc, zc), zc));
+                }
         }
-        // floors, then the largest fractional parts (ties to the lower layer) take one more row each
-        long long given = 0;
-        for (int l = 0; l < L; ++l) {
-            if (!p.active[l * B + b]) continue;
-            const double sh = p.share[l * B + b];
-            const int f = (int)floor(sh);
-            p.budgets[l * B + b] = f;
-            given += f;
-            p.share[l * B + b] = __dsub_rn(sh, (double)f);
+        cube = block_sum(cube, s_part);
+        if (tid == 0) {
+            const double pre = __ddiv_rn(n, __dmul_rn(__dsub_rn(n, 1.0), __dsub_rn(n, 2.0)));
+            p.strength[blockIdx.x] = s;
+            p.skewness[blockIdx.x] = sigma > 0.0 ? __dmul_rn(pre, cube) : 0.0;
+            __threadfence();
+            const unsigned t = atomicAdd(p.ticket, 1u);
+            s_is_last = (t == (unsigned)LB - 1);
+            if (s_is_last) { *p.ticket = 0; __threadfence(); }
         }
-        for (long long left = R - given; left > 0; --left) {
-            int best = -1;
-            double best_frac = 0.0;
-            for (int l = 0; l < L; ++l) {
-                if (!p.active[l * B + b]) continue;
-                const double fr = p.share[l * B + b];
-                if (best < 0 || fr > best_frac) { best = l; best_frac = fr; }
-            }
-            if (best < 0) break;
-            p.budgets[best * B + b] += 1;
-            p.active[best * B + b] = 0;
-        }
+        __syncthreads();
+        if (!s_is_last) return;
+    }
+
+    // ---------------- the last CTA: allocation for every sequence, then the offsets ----------------
+    double *st = reinterpret_cast<double *>(s_dyn);
+    double *sk = st + LB;
+    double *w = sk + LB;
+    double *share = w + LB;
+    int *bud = reinterpret_cast<int *>(share + LB);
+    unsigned char *act = reinterpret_cast<unsigned char *>(bud + LB);
+    for (int i = tid; i < LB; i += kThreads) {
+        st[i] = __ldcg(p.strength + i);
+        sk[i] = __ldcg(p.skewness + i);
     }
     __syncthreads();
+    for (int b = tid >> 5; b < p.B; b += kThreads / 32) allocate_sequence(p, b, st, sk, w, share, act, bud);
+    __syncthreads();
 
-    // ---- offsets: exclusive scan of (budget + Nt + slack) over r = l*B + b ----
-    __shared__ long long s_warp[kAllocThreads / 32];
-    const int n = L * B;
-    const int per = (n + kAllocThreads - 1) / kAllocThreads;
-    const int i0 = threadIdx.x * per, i1 = min(n, i0 + per);
+    // offsets: exclusive scan of (budget + Nt + slack) over r = l*B + b
+    __shared__ long long s_warp[kThreads / 32];
+    const int per = (LB + kThreads - 1) / kThreads;
+    const int i0 = min(LB, tid * per), i1 = min(LB, i0 + per);
     long long local = 0;
-    for (int i = i0; i < i1; ++i) local += p.budgets[i] + p.Nt + p.slack;
+    for (int i = i0; i < i1; ++i) local += bud[i] + p.Nt + p.slack;
     long long incl = local;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = tid & 31, warp = tid >> 5;
 #pragma unroll
     for (int sh = 1; sh < 32; sh <<= 1) {
         const long long o = __shfl_up_sync(0xffffffffu, incl, sh);
@@ -169,22 +239,23 @@ __global__ void __launch_bounds__(kAllocThreads) allocate_kernel(AllocParams p) 
     if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-        long long v = s_warp[lane];
+        long long vv = lane < kThreads / 32 ? s_warp[lane] : 0;
 #pragma unroll
         for (int sh = 1; sh < 32; sh <<= 1) {
-            const long long o = __shfl_up_sync(0xffffffffu, v, sh);
-            if (lane >= sh) v += o;
+            const long long o = __shfl_up_sync(0xffffffffu, vv, sh);
+            if (lane >= sh) vv += o;
         }
-        s_warp[lane] = v;
+        if (lane < kThreads / 32) s_warp[lane] = vv;
     }
     __syncthreads();
     long long run = incl - local + (warp > 0 ? s_warp[warp - 1] : 0);
     for (int i = i0; i < i1; ++i) {
         p.offsets[i] = run;
-        p.lens[i] = p.budgets[i] + p.Nt;
-        run += p.budgets[i] + p.Nt + p.slack;
+        p.lens[i] = bud[i] + p.Nt;
+        p.budgets[i] = bud[i];
+        run += bud[i] + p.Nt + p.slack;
     }
-    if (threadIdx.x == kAllocThreads - 1) p.offsets[n] = s_warp[kAllocThreads / 32 - 1];
+    if (tid == kThreads - 1) p.offsets[LB] = s_warp[kThreads / 32 - 1];
 }
 
 }  // namespace
@@ -193,21 +264,19 @@ int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, 
                   double *strength, double *skewness, aircache_ragged_t *layout, void *ws, cudaStream_t st) {
     const WsLayout w = ws_layout(s);
     const int LB = s->n_layers * s->batch;
-    double *d_st = strength ? strength : ws_ptr<double>(ws, w.mom_strength);
-    double *d_sk = skewness ? skewness : ws_ptr<double>(ws, w.mom_skew);
-    moments_kernel<<<LB, kMomThreads, 0, st>>>(scores, s->n_visual, d_st, d_sk);
-    AIRCACHE_LAUNCH_CHECK();
-    AllocParams p;
-    p.strength = d_st; p.skewness = d_sk;
-    p.w = ws_ptr<double>(ws, w.alloc_w);
-    p.share = ws_ptr<double>(ws, w.alloc_share);
-    p.active = ws_ptr<int32_t>(ws, w.alloc_active);
+    BudgetParams p;
+    p.scores = scores;
+    p.strength = strength ? strength : ws_ptr<double>(ws, w.mom_strength);
+    p.skewness = skewness ? skewness : ws_ptr<double>(ws, w.mom_skew);
     p.budgets = budgets;
     p.offsets = layout->offsets;
     p.lens = layout->lens;
+    p.ticket = ws_ptr<uint32_t>(ws, w.status) + 2;   // second word pair of the status block
     p.L = s->n_layers; p.B = s->batch; p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack; p.mode = mode;
     p.total_kept = kept_per_sequence(s, ratio);
-    allocate_kernel<<<1, kAllocThreads, 0, st>>>(p);
+    const size_t smem = (size_t)LB * (4 * 8 + 4 + 1) + 16;
+    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+    budget_kernel<<<LB, kThreads, smem, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }

@@ -80,9 +80,15 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
         for (int i = threadIdx.x; i < 256; i += kSelThreads) s_hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = s_prefix;
-        for (int i = threadIdx.x; i < n_visual; i += kSelThreads) {
-            const uint32_t key = key_at(i);
-            if ((key & mask) == prefix) atomicAdd(&s_hist[(key >> shift) & 255], 1);
+        // scores of one layer share most of their exponent, so the first passes put nearly every key into one
+        // or two bins: equal digits inside a warp are counted first and added with one atomic
+        for (int i0 = 0; i0 < n_visual; i0 += kSelThreads) {
+            const int i = i0 + threadIdx.x;
+            const uint32_t key = i < n_visual ? key_at(i) : 0u;
+            const bool in = i < n_visual && (key & mask) == prefix;
+            const int bin = in ? (int)((key >> shift) & 255) : -1;
+            const unsigned peers = __match_any_sync(0xffffffffu, bin);
+            if (in && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[bin], __popc(peers));
         }
         __syncthreads();
         if (threadIdx.x < 32) {

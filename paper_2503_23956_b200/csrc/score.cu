@@ -36,6 +36,9 @@ struct ScoreParams {
     int cap, chunks, chunk_keys;
     float scale, sl2, ln_alpha;
     int keep_all;
+    // one launch of the two passes handles the KV groups with rows_lo < elite rows <= rows_hi; the second
+    // launch of a pair adds to the scores the first one wrote
+    int rows_lo, rows_hi, accumulate;
 };
 
 constexpr float kNegBig = -1.0e30f;
@@ -57,13 +60,22 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     const uint16_t *k_cand = k_g + (int64_t)(N - p.W) * p.s_token;
     const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * p.d;
 
-    // Eq. 4, last row only: logit of candidate w for head hl, fp64 dot product in element order.
+    // Eq. 4, last row only: logit of candidate w for head hl, fp64 dot product in element order
+    // (16-byte loads, the eight products of a load are added in order).
     for (int idx = threadIdx.x; idx < p.G * p.W; idx += blockDim.x) {
         const int hl = idx / p.W, w = idx % p.W;
-        const uint16_t *q = q_lb + ((int64_t)(p.W - 1) * p.Hq + g * p.G + hl) * p.d;
-        const uint16_t *kk = k_cand + (int64_t)w * p.s_token;
+        const uint4 *q = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)(p.W - 1) * p.Hq + g * p.G + hl) * p.d);
+        const uint4 *kk = reinterpret_cast<const uint4 *>(k_cand + (int64_t)w * p.s_token);
         double acc = 0.0;
-        for (int c = 0; c < p.d; ++c) acc = __dadd_rn(acc, __dmul_rn((double)bf16_to_f32(q[c]), (double)bf16_to_f32(kk[c])));
+        for (int c = 0; c < p.d / 8; ++c) {
+            const uint4 a = __ldg(q + c), b = __ldg(kk + c);
+            const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc = __dadd_rn(acc, __dmul_rn((double)bf16lo(av[e]), (double)bf16lo(bv[e])));
+                acc = __dadd_rn(acc, __dmul_rn((double)bf16hi(av[e]), (double)bf16hi(bv[e])));
+            }
+        }
         s_logit[idx] = __fmul_rn((float)acc, p.scale);
     }
     __syncthreads();
@@ -110,13 +122,15 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
             if (!((mask >> w2) & 1)) continue;
-            const uint16_t *kk = k_cand + (int64_t)w2 * p.s_token;
+            const uint4 *kk = reinterpret_cast<const uint4 *>(k_cand + (int64_t)w2 * p.s_token);
+            const uint4 *qq = reinterpret_cast<const uint4 *>(q);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            for (int c = 0; c < p.d; c += 4) {
-                a0 = fmaf(bf16_to_f32(q[c]), bf16_to_f32(kk[c]), a0);
-                a1 = fmaf(bf16_to_f32(q[c + 1]), bf16_to_f32(kk[c + 1]), a1);
-                a2 = fmaf(bf16_to_f32(q[c + 2]), bf16_to_f32(kk[c + 2]), a2);
-                a3 = fmaf(bf16_to_f32(q[c + 3]), bf16_to_f32(kk[c + 3]), a3);
+            for (int c = 0; c < p.d / 8; ++c) {
+                const uint4 a = __ldg(qq + c), b = __ldg(kk + c);
+                a0 = fmaf(bf16lo(a.x), bf16lo(b.x), a0); a1 = fmaf(bf16hi(a.x), bf16hi(b.x), a1);
+                a2 = fmaf(bf16lo(a.y), bf16lo(b.y), a2); a3 = fmaf(bf16hi(a.y), bf16hi(b.y), a3);
+                a0 = fmaf(bf16lo(a.z), bf16lo(b.z), a0); a1 = fmaf(bf16hi(a.z), bf16hi(b.z), a1);
+                a2 = fmaf(bf16lo(a.w), bf16lo(b.w), a2); a3 = fmaf(bf16hi(a.w), bf16hi(b.w), a3);
             }
             merge_stats(m, z, ((a0 + a1) + (a2 + a3)) * p.sl2, 1.0f);
         }
@@ -195,6 +209,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
     const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
     const int n_rows = p.row_count[grp];
+    if (n_rows <= p.rows_lo || n_rows > p.rows_hi) return;
     float2 *out = p.chunk_stats + ((int64_t)grp * p.chunks + chunk) * p.cap;
 
     for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
@@ -207,12 +222,18 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = kNegBig; z[nt][0] = z[nt][1] = 0.f; }
 
+        // software pipeline: the next tile's keys are requested before this tile's MMAs
+        auto fetch = [&](KeyFrag<D> &dst, int kt) {
+            const int ka = kt + gid, kb = kt + gid + 8;
+            load_keys<D>(dst, k_g + (int64_t)(ka < key1 ? ka : key1 - 1) * p.s_token,
+                         k_g + (int64_t)(kb < key1 ? kb : key1 - 1) * p.s_token, t);
+        };
+        KeyFrag<D> f, f_next;
+        if (key0 + warp * 16 < key1) fetch(f, key0 + warp * 16);
         for (int kt = key0 + warp * 16; kt < key1; kt += 64) {
             const int ka = kt + gid, kb = kt + gid + 8;
             const bool va = ka < key1, vb = kb < key1;
-            KeyFrag<D> f;
-            load_keys<D>(f, k_g + (int64_t)(va ? ka : key1 - 1) * p.s_token,
-                         k_g + (int64_t)(vb ? kb : key1 - 1) * p.s_token, t);
+            if (kt + 64 < key1) fetch(f_next, kt + 64);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 if (nt < nt_used) {
@@ -230,6 +251,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
                     }
                 }
             }
+            if (kt + 64 < key1) f = f_next;
         }
         // combine the eight key lanes of a column, then the four warps, in a fixed order
 #pragma unroll
@@ -270,11 +292,14 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
     const int kbase = blockIdx.x * kScoreKeyTile + warp * 32;
     float imp[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [m-tile][key gid / gid+8]
+    bool any = false;
 
     for (int g = 0; g < p.Hkv; ++g) {
         const int grp = lb * p.Hkv + g;
         const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
         const int n_rows = p.row_count[grp];
+        if (n_rows <= p.rows_lo || n_rows > p.rows_hi) continue;
+        any = true;
         KeyFrag<D> f[2];
         bool valid[2][2];
 #pragma unroll
@@ -318,6 +343,7 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
             }
         }
     }
+    if (p.accumulate && !any) return;
     float *out = p.scores + (int64_t)lb * p.Nv;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
@@ -327,14 +353,15 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
             v += __shfl_xor_sync(0xffffffffu, v, 1);
             v += __shfl_xor_sync(0xffffffffu, v, 2);
             const int key = kbase + mt * 16 + gid + 8 * j;
-            if (t == 0 && key < p.Nv) out[key] = v;
+            if (t == 0 && key < p.Nv) out[key] = p.accumulate ? out[key] + v : v;
         }
     }
 }
 
 template <int D, int NT>
-int launch_passes(const ScoreParams &p, cudaStream_t st) {
+int launch_passes(ScoreParams p, int rows_lo, int rows_hi, int accumulate, cudaStream_t st) {
     const int64_t LB = (int64_t)p.L * p.B;
+    p.rows_lo = rows_lo; p.rows_hi = rows_hi; p.accumulate = accumulate;
     stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)(LB * p.Hkv)), 128, 0, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)LB), 128, 0, st>>>(p);
@@ -342,13 +369,20 @@ int launch_passes(const ScoreParams &p, cudaStream_t st) {
     return AIRCACHE_OK;
 }
 
+// The number of elite rows of a KV group is known on the device only and is small for the paper's
+// threshold (a few rows per head), far below the G*W the shape allows.  Groups with at most 32 rows run in
+// a 4-tile instantiation (few registers, more CTAs per SM); if the shape allows more rows, a second pair of
+// launches with the wide instantiation picks up the groups beyond 32 rows and exits at once elsewhere.
 template <int D>
 int launch_passes_d(const ScoreParams &p, cudaStream_t st) {
     const int nt_max = (p.G * p.W + 7) / 8;
-    if (nt_max <= 2) return launch_passes<D, 2>(p, st);
-    if (nt_max <= 4) return launch_passes<D, 4>(p, st);
-    if (nt_max <= 8) return launch_passes<D, 8>(p, st);
-    return launch_passes<D, 16>(p, st);
+    const int big = 1 << 30;
+    if (nt_max <= 2) return launch_passes<D, 2>(p, 0, big, 0, st);
+    if (nt_max <= 4) return launch_passes<D, 4>(p, 0, big, 0, st);
+    int rc = launch_passes<D, 4>(p, 0, 32, 0, st);
+    if (rc) return rc;
+    if (nt_max <= 8) return launch_passes<D, 8>(p, 32, big, 1, st);
+    return launch_passes<D, 16>(p, 32, big, 1, st);
 }
 
 }  // namespace
