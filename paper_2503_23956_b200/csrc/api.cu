@@ -66,6 +66,8 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.row_coef = take(groups * cap * 4);
     w.row_text = take(groups * cap * 8);
     w.chunk_stats = take(groups * chunks * cap * 8);
+    w.row_final = take(groups * cap * 8);
+    w.group_ticket = take(groups * 4);
     w.mom_strength = take(LB * 8);
     w.mom_skew = take(LB * 8);
     w.alloc_w = take(LB * 8);

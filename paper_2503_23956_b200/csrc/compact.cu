@@ -81,14 +81,19 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
         __syncthreads();
         const uint32_t prefix = s_prefix;
         // scores of one layer share most of their exponent, so the first passes put nearly every key into one
-        // or two bins: equal digits inside a warp are counted first and added with one atomic
+        // or two bins: a warp whose 32 keys share the digit adds them with one atomic
         for (int i0 = 0; i0 < n_visual; i0 += kSelThreads) {
             const int i = i0 + threadIdx.x;
             const uint32_t key = i < n_visual ? key_at(i) : 0u;
             const bool in = i < n_visual && (key & mask) == prefix;
             const int bin = in ? (int)((key >> shift) & 255) : -1;
-            const unsigned peers = __match_any_sync(0xffffffffu, bin);
-            if (in && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[bin], __popc(peers));
+            int same;
+            __match_all_sync(0xffffffffu, bin, &same);
+            if (same) {
+                if (in && (threadIdx.x & 31) == 0) atomicAdd(&s_hist[bin], 32);
+            } else if (in) {
+                atomicAdd(&s_hist[bin], 1);
+            }
         }
         __syncthreads();
         if (threadIdx.x < 32) {

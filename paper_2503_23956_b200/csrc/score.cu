@@ -1,18 +1,23 @@
 // aircache_score: importance of every visual token seen from the elite observation window
 // (Section 3.3, Eq. 4-8), all layers and sequences per launch.
 //
-// Three kernels on one stream:
-//   elite_kernel       one CTA per (layer, sequence, KV head): Eq. 4 logits of the last text query against
-//                      the W candidate keys (fp64 dot products, so the Eq. 5 decision does not depend on a
-//                      summation order), the elite set of each query head, the list of elite rows
-//                      (head, window slot) of the KV group, and each row's softmax statistics over the
-//                      text keys it may see (elite, causal).
+// Kernels on one stream:
+//   elite_kernel       one CTA per (layer, sequence, KV head): the W candidate keys and the last text query
+//                      are staged in shared memory; Eq. 4 logits as fp64 dot products in element order (so
+//                      the Eq. 5 decision does not depend on a summation order), the elite set of each
+//                      query head, the table of elite rows (head, window slot) of the KV group, and each
+//                      row's softmax statistics over the text keys it may see (elite, causal).
 //   stats_kernel       Eq. 7 pass one: Q_tk K_v^T on tensor cores (keys on the M axis, elite rows on N),
-//                      running (max, sum of exp2) of every elite row over one chunk of visual keys.
-//   importance_kernel  Eq. 7 pass two + Eq. 8: recomputes the same tiles (keys now come from L2), turns
-//                      logits into probabilities with the merged statistics and sums the rows of all heads
-//                      per key with weight 1 / (|E_h| Hq).  KV heads are visited in ascending order by one
-//                      thread per key, so the sum has a fixed order.
+//                      running (max, sum of exp2) of every elite row over one chunk of visual keys.  The CTA
+//                      that finishes a KV group last (ticket) merges the chunks and the text statistics
+//                      into one (max, weight / normaliser) pair per row.
+//   importance_kernel  Eq. 7 pass two + Eq. 8: recomputes the same tiles (keys now come from L2 when the
+//                      cache is small enough), turns logits into probabilities and sums the rows of all
+//                      heads per key with weight 1 / (|E_h| Hq).  KV heads are visited in ascending order
+//                      by one thread per key, so the sum has a fixed order.
+//
+// Both passes read the keys straight from global memory into MMA fragments: every key byte is used once
+// per CTA, so staging it in shared memory would only add a round trip.
 #include <math.h>
 
 #include "common.cuh"
@@ -32,13 +37,14 @@ struct ScoreParams {
     float *row_coef;
     float2 *row_text;
     float2 *chunk_stats;
+    float2 *row_final;   // (max, weight / normaliser) per elite row, written by the last stats CTA of a group
+    uint32_t *group_ticket;
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
     int cap, chunks, chunk_keys;
     float scale, sl2, ln_alpha;
     int keep_all;
-    // one launch of the two passes handles the KV groups with rows_lo < elite rows <= rows_hi; the second
-    // launch of a pair adds to the scores the first one wrote
-    int rows_lo, rows_hi, accumulate;
+    // one stats launch handles the KV groups with rows_lo < elite rows <= rows_hi
+    int rows_lo, rows_hi;
 };
 
 constexpr float kNegBig = -1.0e30f;
@@ -46,7 +52,12 @@ constexpr float kNegBig = -1.0e30f;
 // ---------------------------------------------------------------------------------------------
 // Eq. 4-5 and the elite-row table
 // ---------------------------------------------------------------------------------------------
+template <int D>
 __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
+    constexpr int KS = D + 8;   // padded row: 16-byte reads of consecutive rows fall into different banks
+    extern __shared__ __align__(16) uint16_t s_dyn[];
+    uint16_t *s_k = s_dyn;                 // [W][KS]   candidate keys
+    uint16_t *s_ql = s_dyn + p.W * KS;     // [G][KS]   queries of the last text token
     __shared__ float s_logit[kMaxGroup * kMaxWindow];
     __shared__ uint64_t s_mask[kMaxGroup];
     __shared__ int s_first_row[kMaxGroup + 1];
@@ -58,18 +69,27 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     const int N = p.Nv + p.Nt;
     const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
     const uint16_t *k_cand = k_g + (int64_t)(N - p.W) * p.s_token;
-    const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * p.d;
+    const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * D;
 
-    // Eq. 4, last row only: logit of candidate w for head hl, fp64 dot product in element order
-    // (16-byte loads, the eight products of a load are added in order).
+    if (threadIdx.x == 0) p.group_ticket[grp] = 0;   // the statistics pass counts its chunks here
+    for (int idx = threadIdx.x; idx < (p.W + p.G) * (D / 8); idx += blockDim.x) {
+        const int row = idx / (D / 8), c = idx % (D / 8);
+        const uint16_t *src = row < p.W ? k_cand + (int64_t)row * p.s_token
+                                        : q_lb + ((int64_t)(p.W - 1) * p.Hq + g * p.G + (row - p.W)) * D;
+        *reinterpret_cast<uint4 *>(s_dyn + row * KS + c * 8) = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+    }
+    __syncthreads();
+
+    // Eq. 4, last row only: logit of candidate w for head hl, fp64 dot product in element order.
     for (int idx = threadIdx.x; idx < p.G * p.W; idx += blockDim.x) {
         const int hl = idx / p.W, w = idx % p.W;
-        const uint4 *q = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)(p.W - 1) * p.Hq + g * p.G + hl) * p.d);
-        const uint4 *kk = reinterpret_cast<const uint4 *>(k_cand + (int64_t)w * p.s_token);
+        const uint4 *q = reinterpret_cast<const uint4 *>(s_ql + hl * KS);
+        const uint4 *kk = reinterpret_cast<const uint4 *>(s_k + w * KS);
         double acc = 0.0;
-        for (int c = 0; c < p.d / 8; ++c) {
-            const uint4 a = __ldg(q + c), b = __ldg(kk + c);
-            const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll 4
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 a = q[c], bb = kk[c];
+            const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 acc = __dadd_rn(acc, __dmul_rn((double)bf16lo(av[e]), (double)bf16lo(bv[e])));
@@ -117,20 +137,24 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         const int r = s_first_row[hl] + __popcll(mask & (((uint64_t)1 << w) - 1));
         info[r] = (hl << 8) | w;
         coef[r] = 1.0f / ((float)__popcll(mask) * (float)p.Hq);
-        // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.
-        const uint16_t *q = q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * p.d;
+        // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.  The query row goes to registers
+        // once, the keys come from shared memory.
+        uint4 qr[D / 8];
+        const uint4 *qq = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
             if (!((mask >> w2) & 1)) continue;
-            const uint4 *kk = reinterpret_cast<const uint4 *>(k_cand + (int64_t)w2 * p.s_token);
-            const uint4 *qq = reinterpret_cast<const uint4 *>(q);
+            const uint4 *kk = reinterpret_cast<const uint4 *>(s_k + w2 * KS);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            for (int c = 0; c < p.d / 8; ++c) {
-                const uint4 a = __ldg(qq + c), b = __ldg(kk + c);
-                a0 = fmaf(bf16lo(a.x), bf16lo(b.x), a0); a1 = fmaf(bf16hi(a.x), bf16hi(b.x), a1);
-                a2 = fmaf(bf16lo(a.y), bf16lo(b.y), a2); a3 = fmaf(bf16hi(a.y), bf16hi(b.y), a3);
-                a0 = fmaf(bf16lo(a.z), bf16lo(b.z), a0); a1 = fmaf(bf16hi(a.z), bf16hi(b.z), a1);
-                a2 = fmaf(bf16lo(a.w), bf16lo(b.w), a2); a3 = fmaf(bf16hi(a.w), bf16hi(b.w), a3);
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) {
+                const uint4 a = qr[c], bb = kk[c];
+                a0 = fmaf(bf16lo(a.x), bf16lo(bb.x), a0); a1 = fmaf(bf16hi(a.x), bf16hi(bb.x), a1);
+                a2 = fmaf(bf16lo(a.y), bf16lo(bb.y), a2); a3 = fmaf(bf16hi(a.y), bf16hi(bb.y), a3);
+                a0 = fmaf(bf16lo(a.z), bf16lo(bb.z), a0); a1 = fmaf(bf16hi(a.z), bf16hi(bb.z), a1);
+                a2 = fmaf(bf16lo(a.w), bf16lo(bb.w), a2); a3 = fmaf(bf16hi(a.w), bf16hi(bb.w), a3);
             }
             merge_stats(m, z, ((a0 + a1) + (a2 + a3)) * p.sl2, 1.0f);
         }
@@ -198,6 +222,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
     constexpr int QS = D + 32;
     __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
     __shared__ float2 s_red[4][NT * 8];
+    __shared__ int s_is_last;
 
     const int grp = blockIdx.y;
     const int g = grp % p.Hkv;
@@ -275,8 +300,37 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
             float2 a = s_red[0][r];
 #pragma unroll
             for (int w2 = 1; w2 < 4; ++w2) merge_stats(a.x, a.y, s_red[w2][r].x, s_red[w2][r].y);
-            if (row0 + r < n_rows) out[row0 + r] = a;
+            if (row0 + r < n_rows) __stcg(out + row0 + r, a);
         }
+    }
+
+    // The CTA that finishes the group last merges text and chunk statistics, one warp per row: lanes take
+    // chunks lane, lane + 32, ... in order, then a fixed xor tree.  (The ticket was zeroed by elite_kernel.)
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s_is_last = atomicAdd(p.group_ticket + grp, 1u) == (unsigned)p.chunks - 1;
+        if (s_is_last) __threadfence();
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    for (int r = warp; r < n_rows; r += 4) {
+        float mm = kNegBig, zz = 0.f;
+        if (lane == 0) {
+            const float2 tx = p.row_text[(int64_t)grp * p.cap + r];
+            mm = tx.x; zz = tx.y;
+        }
+        for (int c = lane; c < p.chunks; c += 32) {
+            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)grp * p.chunks + c) * p.cap + r);
+            merge_stats(mm, zz, cs.x, cs.y);
+        }
+#pragma unroll
+        for (int sh = 1; sh < 32; sh <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mm, sh);
+            const float z2 = __shfl_xor_sync(0xffffffffu, zz, sh);
+            merge_stats(mm, zz, m2, z2);
+        }
+        if (lane == 0) p.row_final[(int64_t)grp * p.cap + r] = make_float2(mm, p.row_coef[(int64_t)grp * p.cap + r] / zz);
     }
 }
 
@@ -292,41 +346,24 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
     const int kbase = blockIdx.x * kScoreKeyTile + warp * 32;
     float imp[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [m-tile][key gid / gid+8]
-    bool any = false;
 
     for (int g = 0; g < p.Hkv; ++g) {
         const int grp = lb * p.Hkv + g;
         const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
         const int n_rows = p.row_count[grp];
-        if (n_rows <= p.rows_lo || n_rows > p.rows_hi) continue;
-        any = true;
         KeyFrag<D> f[2];
-        bool valid[2][2];
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
             const int ka = kbase + mt * 16 + gid, kb = ka + 8;
-            valid[mt][0] = ka < p.Nv;
-            valid[mt][1] = kb < p.Nv;
-            load_keys<D>(f[mt], k_g + (int64_t)(valid[mt][0] ? ka : p.Nv - 1) * p.s_token,
-                         k_g + (int64_t)(valid[mt][1] ? kb : p.Nv - 1) * p.s_token, t);
+            load_keys<D>(f[mt], k_g + (int64_t)(ka < p.Nv ? ka : p.Nv - 1) * p.s_token,
+                         k_g + (int64_t)(kb < p.Nv ? kb : p.Nv - 1) * p.s_token, t);
         }
         for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
             const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
             __syncthreads();
             stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
-            for (int r = threadIdx.x; r < nt_used * 8; r += blockDim.x) {
-                float2 st = make_float2(0.f, 0.f);
-                if (row0 + r < n_rows) {
-                    const float2 tx = p.row_text[(int64_t)grp * p.cap + row0 + r];
-                    float m = tx.x, z = tx.y;
-                    for (int c = 0; c < p.chunks; ++c) {
-                        const float2 cs = p.chunk_stats[((int64_t)grp * p.chunks + c) * p.cap + row0 + r];
-                        merge_stats(m, z, cs.x, cs.y);
-                    }
-                    st = make_float2(m, p.row_coef[(int64_t)grp * p.cap + row0 + r] / z);
-                }
-                s_stat[r] = st;
-            }
+            for (int r = threadIdx.x; r < nt_used * 8; r += blockDim.x)
+                s_stat[r] = row0 + r < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + r] : make_float2(0.f, 0.f);
             __syncthreads();
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
@@ -343,7 +380,6 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
             }
         }
     }
-    if (p.accumulate && !any) return;
     float *out = p.scores + (int64_t)lb * p.Nv;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
@@ -353,36 +389,47 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
             v += __shfl_xor_sync(0xffffffffu, v, 1);
             v += __shfl_xor_sync(0xffffffffu, v, 2);
             const int key = kbase + mt * 16 + gid + 8 * j;
-            if (t == 0 && key < p.Nv) out[key] = p.accumulate ? out[key] + v : v;
+            if (t == 0 && key < p.Nv) out[key] = v;
         }
     }
 }
 
 template <int D, int NT>
-int launch_passes(ScoreParams p, int rows_lo, int rows_hi, int accumulate, cudaStream_t st) {
-    const int64_t LB = (int64_t)p.L * p.B;
-    p.rows_lo = rows_lo; p.rows_hi = rows_hi; p.accumulate = accumulate;
-    stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)(LB * p.Hkv)), 128, 0, st>>>(p);
+int launch_stats(ScoreParams p, int rows_lo, int rows_hi, cudaStream_t st) {
+    p.rows_lo = rows_lo; p.rows_hi = rows_hi;
+    stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)((int64_t)p.L * p.B * p.Hkv)), 128, 0, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
-    importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)LB), 128, 0, st>>>(p);
+    return AIRCACHE_OK;
+}
+
+template <int D, int NT>
+int launch_importance(const ScoreParams &p, cudaStream_t st) {
+    importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)((int64_t)p.L * p.B)), 128, 0,
+                               st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }
 
 // The number of elite rows of a KV group is known on the device only and is small for the paper's
-// threshold (a few rows per head), far below the G*W the shape allows.  Groups with at most 32 rows run in
-// a 4-tile instantiation (few registers, more CTAs per SM); if the shape allows more rows, a second pair of
-// launches with the wide instantiation picks up the groups beyond 32 rows and exits at once elsewhere.
+// threshold (a few rows per head), far below the G*W the shape allows.  The statistics pass keeps per-row
+// state in registers, so groups with at most 32 rows run in a 4-tile instantiation (more CTAs per SM); if
+// the shape allows more rows, a second launch with the wide instantiation picks up the groups beyond 32
+// rows and exits at once elsewhere.  The importance pass keeps no per-row state and runs once.
 template <int D>
 int launch_passes_d(const ScoreParams &p, cudaStream_t st) {
     const int nt_max = (p.G * p.W + 7) / 8;
     const int big = 1 << 30;
-    if (nt_max <= 2) return launch_passes<D, 2>(p, 0, big, 0, st);
-    if (nt_max <= 4) return launch_passes<D, 4>(p, 0, big, 0, st);
-    int rc = launch_passes<D, 4>(p, 0, 32, 0, st);
-    if (rc) return rc;
-    if (nt_max <= 8) return launch_passes<D, 8>(p, 32, big, 1, st);
-    return launch_passes<D, 16>(p, 32, big, 1, st);
+    int rc;
+    if (nt_max <= 2) {
+        if ((rc = launch_stats<D, 2>(p, 0, big, st))) return rc;
+        return launch_importance<D, 2>(p, st);
+    }
+    if ((rc = launch_stats<D, 4>(p, 0, nt_max <= 4 ? big : 32, st))) return rc;
+    if (nt_max > 4) {
+        rc = nt_max <= 8 ? launch_stats<D, 8>(p, 32, big, st) : launch_stats<D, 16>(p, 32, big, st);
+        if (rc) return rc;
+    }
+    return nt_max <= 4 ? launch_importance<D, 4>(p, st) : launch_importance<D, 8>(p, st);
 }
 
 }  // namespace
@@ -401,6 +448,8 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.row_coef = ws_ptr<float>(ws, w.row_coef);
     p.row_text = ws_ptr<float2>(ws, w.row_text);
     p.chunk_stats = ws_ptr<float2>(ws, w.chunk_stats);
+    p.row_final = ws_ptr<float2>(ws, w.row_final);
+    p.group_ticket = ws_ptr<uint32_t>(ws, w.group_ticket);
     p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
     p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
     p.cap = score_row_cap(s);
@@ -410,9 +459,12 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.sl2 = s->scale * kLog2e;
     p.keep_all = alpha <= 0.0f;
     p.ln_alpha = p.keep_all ? 0.0f : (float)log((double)alpha);
+    p.rows_lo = 0; p.rows_hi = 1 << 30;
 
     const int64_t groups = (int64_t)p.L * p.B * p.Hkv;
-    elite_kernel<<<(unsigned)groups, 128, 0, st>>>(p);
+    const size_t elite_smem = (size_t)(p.W + p.G) * (p.d + 8) * 2;
+    if (s->head_dim == 64) elite_kernel<64><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+    else elite_kernel<128><<<(unsigned)groups, 128, elite_smem, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     return s->head_dim == 64 ? launch_passes_d<64>(p, st) : launch_passes_d<128>(p, st);
 }
