@@ -16,6 +16,8 @@ layers of a real model.
                   call / average duration of a call inside the timed region
   e2e             the same metric through aircache_pipeline_host: pinned host inputs, host outputs
   cpu_baseline    the CPU oracle timed on this host (rank 0, N = 1 only)
+  hbm_bound_workloads   the decode and compaction rooflines on further workloads (default: config 4, 261 MB
+                  per decode launch), measured briefly after the main run at N = 1
 
 `python bench.py --impl reference` times the CPU oracle instead (there is no other implementation of the
 paper's method to run).  Under torchrun every rank runs the same workload on its own GPU with its own seeds
@@ -60,6 +62,8 @@ def parse_args():
     ap.add_argument("--decode-steps", type=int, default=0, help="decode rounds per step (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--extra", default="c4", help="comma list of further workloads measured briefly at N = 1 "
+                                                  "(decode and compaction rooflines); empty string to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -165,32 +169,13 @@ def decode_cu_sha1():
     return hashlib.sha1(open(p, "rb").read()).hexdigest()[:12]
 
 
-def run_cuda(args):
-    import paper_2503_23956_b200 as ac
+def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist):
+    """Times `steps` steps of the whole path on `rotate` resident request batches of workload `wl`.
+    Returns (local numbers, the sessions) -- the caller reduces over ranks."""
     from paper_2503_23956_b200.session import Session
     from workloads import decode_queries, full_cache, window_queries
 
-    rank, local_rank, world = dist_info()
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the AirCache path has no CPU fallback")
-    dev = torch.device("cuda", local_rank)
-    torch.cuda.set_device(dev)
-    ac.lib()  # fail loudly if the library is missing
-
-    wl = pick_workload(args.workload, args.ratio)
-    n_dec = args.decode_steps or wl.steps
     sh = shape_of(ac, wl)
-    row_bytes = wl.n_kv_heads * wl.head_dim * 2
-    T = ac.aircache_kept_per_sequence(sh, wl.ratio)
-    cache_bytes = 2 * row_bytes * wl.batch * (T + wl.n_layers * wl.n_text)   # K' + V' valid rows of one request batch
-    rotate = args.rotate or max(2, -(-2 * L2_BYTES // cache_bytes))
-    rotate = min(rotate, 16)
-
-    # ---- resident inputs: `rotate` independent request batches ----
     reqs = []
     for i in range(rotate):
         w = wl.with_(seed=wl.seed + 1000 * rank + i)
@@ -202,9 +187,7 @@ def run_cuda(args):
         s.out_steps = torch.empty((n_dec,) + tuple(s.out.shape), dtype=torch.float32, device=dev)
         reqs.append(s)
     torch.cuda.synchronize()
-
     stream = torch.cuda.Stream(device=dev)
-    launches = {"score": 3, "budget": 2, "compact": 2, "decode": 1}   # kernels per C-ABI call
 
     def stage_score():
         for s in reqs:
@@ -229,7 +212,7 @@ def run_cuda(args):
         for _, fn in stages[:3]:
             fn()       # one eager pass: the compressed caches exist before the decode graph is captured
         stream.synchronize()
-        if not args.no_graph:
+        if use_graph:
             for name, fn in stages:
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=stream):
@@ -249,14 +232,14 @@ def run_cuda(args):
         return [torch.cuda.Event(enable_timing=True) for _ in range(5)]
 
     with torch.cuda.stream(stream):
-        for _ in range(max(args.warmup, 3)):
+        for _ in range(warmup):
             run_step(new_events())
         stream.synchronize()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-        sampler = ClockSampler(local_rank)
-        evs = [new_events() for _ in range(args.steps)]
+        sampler = ClockSampler(dev.index or 0)
+        evs = [new_events() for _ in range(steps)]
         for e in evs:
             run_step(e)
         torch.cuda.synchronize()
@@ -266,59 +249,124 @@ def run_cuda(args):
     for s in reqs:
         if s.status() != 0:
             raise RuntimeError("a device-side wait timed out")
-
     total_ms = evs[0][0].elapsed_time(evs[-1][4])
-    stage_ms = {name: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / args.steps
-                for i, (name, _) in enumerate(stages)}
-    tokens_per_step = rotate * n_dec * wl.batch
-    total_ms_all, tokens_all = reduce_over_ranks(total_ms, tokens_per_step * args.steps, dev, dist)
-    decode_ms_all, _ = reduce_over_ranks(stage_ms["decode"], 0, dev, dist)
-
-    # ---- roofline of the dominant kernel (decode attention) ----
+    stage_ms = {name: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / steps for i, (name, _) in enumerate(stages)}
     valid_rows = sum(int(s.lens.sum().item()) for s in reqs) / rotate
+    return dict(total_ms=total_ms, stage_ms=stage_ms, clocks=clocks, valid_rows=valid_rows, graph=bool(graphs)), reqs
+
+
+def rooflines(ac, wl, m, rotate, n_dec, traffic=None):
+    """Decode-attention and compaction rooflines from one measurement (algorithmic bytes / measured time)."""
+    sh = shape_of(ac, wl)
+    row_bytes = wl.n_kv_heads * wl.head_dim * 2
+    T = ac.aircache_kept_per_sequence(sh, wl.ratio)
     q_out_bytes = wl.n_layers * wl.batch * wl.n_q_heads * wl.head_dim * 6
-    alg_bytes = 2 * row_bytes * valid_rows + q_out_bytes
-    calls = rotate * n_dec
-    call_us = stage_ms["decode"] * 1e3 / calls
+    alg_bytes = 2 * row_bytes * m["valid_rows"] + q_out_bytes
+    call_us = m["stage_ms"]["decode"] * 1e3 / (rotate * n_dec)
     achieved = alg_bytes / (call_us * 1e-6) / 1e9
     peak, peak_kind = measured_peaks()
+    compact_bytes = 2 * alg_bytes - 2 * q_out_bytes + 4 * wl.batch * T     # read + write of every row, indices
+    comp_us = m["stage_ms"]["compact"] * 1e3 / rotate
+    dec = {"kernel": "decode_kernel (one launch per aircache_decode_attn call)", "bound": "hbm",
+           "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+           "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
+           "bytes_per_call": alg_bytes, "us_per_call": call_us}
+    comp = {"kernel": "select_kernel + gather_kernel per aircache_compact call", "bound": "hbm",
+            "achieved": compact_bytes / (comp_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+            "frac": compact_bytes / (comp_us * 1e-6) / 1e9 / peak,
+            "frac_of_8TBs_nominal": compact_bytes / (comp_us * 1e-6) / 1e9 / 8000.0,
+            "bytes_per_call": compact_bytes, "us_per_call": comp_us}
+    return dec, comp
+
+
+def default_rotate(ac, wl):
+    sh = shape_of(ac, wl)
+    T = ac.aircache_kept_per_sequence(sh, wl.ratio)
+    cache_bytes = 2 * wl.n_kv_heads * wl.head_dim * 2 * wl.batch * (T + wl.n_layers * wl.n_text)
+    return min(16, max(2, -(-2 * L2_BYTES // cache_bytes))), cache_bytes
+
+
+def kernels_per_step(wl, rotate, n_dec):
+    """Launches of this library's kernels in one step: elite + statistics (one launch, two when a KV group may
+    have more than 32 elite rows) + importance; budget; select + gather; one decode kernel per call."""
+    nt_max = (wl.group * wl.window + 7) // 8
+    score = 1 + (1 if nt_max <= 4 else 2) + 1
+    return rotate * (score + 1 + 2 + n_dec)
+
+
+def run_cuda(args):
+    import paper_2503_23956_b200 as ac
+
+    rank, local_rank, world = dist_info()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the AirCache path has no CPU fallback")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    ac.lib()  # fail loudly if the library is missing
+
+    wl = pick_workload(args.workload, args.ratio)
+    n_dec = args.decode_steps or wl.steps
+    sh = shape_of(ac, wl)
+    rotate, cache_bytes = default_rotate(ac, wl)
+    rotate = args.rotate or rotate
+    warmup = max(args.warmup, 3)
+    m, reqs = measure(ac, wl, n_dec, rotate, args.steps, warmup, not args.no_graph, dev, rank, dist)
+    stage_ms = m["stage_ms"]
+    tokens_per_step = rotate * n_dec * wl.batch
+    total_ms_all, tokens_all = reduce_over_ranks(m["total_ms"], tokens_per_step * args.steps, dev, dist)
+    decode_ms_all, _ = reduce_over_ranks(stage_ms["decode"], 0, dev, dist)
     traffic = None
     if NCU_TRAFFIC["bytes_per_launch"] and NCU_TRAFFIC["decode_cu_sha1"] == decode_cu_sha1() \
             and NCU_TRAFFIC["workload"] == args.workload and args.ratio is None:
         traffic = NCU_TRAFFIC["bytes_per_launch"]
-    compact_bytes = 2 * alg_bytes - 2 * q_out_bytes + 4 * wl.batch * T     # read + write of every kept row, indices
-    comp_us = stage_ms["compact"] * 1e3 / rotate
+    roof_dec, roof_comp = rooflines(ac, wl, m, rotate, n_dec, traffic)
 
     result = {
         "metric": METRIC, "value": tokens_all / (total_ms_all * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms_all / args.steps,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": total_ms_all / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{wl.name} r={wl.ratio:g} B={wl.batch} L={wl.n_layers} Hq={wl.n_q_heads} "
-                               f"Hkv={wl.n_kv_heads} d={wl.head_dim} Nv={wl.n_visual} Nt={wl.n_text} W={wl.window}",
-                   "decode_steps": n_dec, "resident_requests": rotate,
+        "config": {"workload": describe(wl), "decode_steps": n_dec, "resident_requests": rotate,
                    "l2": f"inputs larger than L2: {rotate} independent requests served round-robin, "
                          f"{rotate * cache_bytes / 2 ** 20:.0f} MiB of compressed cache cycled per decode round",
-                   "launch": "CUDA graph replay of the C-ABI calls" if graphs else "direct C-ABI calls",
+                   "launch": "CUDA graph replay of the C-ABI calls" if m["graph"] else "direct C-ABI calls",
                    "attention_only": True},
         "decode_tok_s": world * tokens_per_step / (decode_ms_all * 1e-3),
         "compress_us_per_layer": (stage_ms["score"] + stage_ms["budget"] + stage_ms["compact"]) * 1e3
                                  / (rotate * wl.n_layers),
         "stage_us_per_request": {k: v * 1e3 / rotate for k, v in stage_ms.items()},
-        "roofline": {"kernel": "decode_kernel (one launch per aircache_decode_attn call)", "bound": "hbm",
-                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
-                     "bytes_per_call": alg_bytes, "us_per_call": call_us},
-        "roofline_compact": {"kernel": "select_kernel + gather_kernel per aircache_compact call", "bound": "hbm",
-                             "achieved": compact_bytes / (comp_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-                             "frac": compact_bytes / (comp_us * 1e-6) / 1e9 / peak, "bytes_per_call": compact_bytes,
-                             "us_per_call": comp_us},
-        "clocks": clocks,
-        "gpu_launches": args.steps * rotate * (launches["score"] + launches["budget"] + launches["compact"]
-                                               + n_dec * launches["decode"]),
+        "roofline": roof_dec,
+        "roofline_compact": roof_comp,
+        "clocks": m["clocks"],
+        "gpu_launches": args.steps * kernels_per_step(wl, rotate, n_dec),
     }
-
     if rank == 0 and not args.no_e2e:
         result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 5))
+    del reqs
+    torch.cuda.empty_cache()
+
+    # The default workload moves 49 MB per decode launch, about 7.6 us of HBM time: launch, prologue and the
+    # split-K merge weigh as much as the stream.  The same kernels on the HBM-bound configurations:
+    if rank == 0 and world == 1 and args.extra:
+        extra = {}
+        for spec in args.extra.split(","):
+            w2 = pick_workload(spec, None)
+            r2, _ = default_rotate(ac, w2)
+            d2 = min(w2.steps, 32)
+            m2, q2 = measure(ac, w2, d2, r2, 3, 3, not args.no_graph, dev, rank, None)
+            dec2, comp2 = rooflines(ac, w2, m2, r2, d2)
+            extra[spec] = {"workload": describe(w2), "decode_steps": d2, "resident_requests": r2,
+                           "decode_tok_s": r2 * d2 * w2.batch / (m2["stage_ms"]["decode"] * 1e-3),
+                           "compress_us_per_layer": (m2["stage_ms"]["score"] + m2["stage_ms"]["budget"] +
+                                                     m2["stage_ms"]["compact"]) * 1e3 / (r2 * w2.n_layers),
+                           "stage_us_per_request": {k: v * 1e3 / r2 for k, v in m2["stage_ms"].items()},
+                           "roofline": dec2, "roofline_compact": comp2, "clocks": m2["clocks"]}
+            del q2
+            torch.cuda.empty_cache()
+        result["hbm_bound_workloads"] = extra
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, n_dec)
     if dist is not None:
@@ -326,6 +374,11 @@ def run_cuda(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(result))
+
+
+def describe(wl):
+    return (f"{wl.name} r={wl.ratio:g} B={wl.batch} L={wl.n_layers} Hq={wl.n_q_heads} Hkv={wl.n_kv_heads} "
+            f"d={wl.head_dim} Nv={wl.n_visual} Nt={wl.n_text} W={wl.window}")
 
 
 def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
@@ -420,9 +473,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{wl.name} r={wl.ratio:g} B={wl.batch} L={wl.n_layers} Hq={wl.n_q_heads} "
-                               f"Hkv={wl.n_kv_heads} d={wl.head_dim} Nv={wl.n_visual} Nt={wl.n_text} W={wl.window}",
-                   "decode_steps": n_dec, "attention_only": True},
+        "config": {"workload": describe(wl), "decode_steps": n_dec, "attention_only": True},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["threads"], "kind": "oracle",
                          "sample": last["sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

@@ -207,10 +207,23 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int n = p.n_regions;
     const int n_ctas = (int)gridDim.x;
+    // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as SMs free up,
+    // and this one does everything that reads no global memory before it waits for its predecessor.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (wid == NCW && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
     }
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&s_bar[s]), 1);             // full: the producer's expect_tx arrival
+            mbar_init(smem_u32(&s_bar[kStages + s]), NCW);  // empty: one arrival per consumer warp
+        }
+        mbar_init(smem_u32(&s_bar[2 * kStages]), 1);        // partials staged for the final merge
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_abort = 0;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- unit prefix and first row of all regions (every CTA computes the same tables) ----
     {
@@ -222,7 +235,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             s_off[i] = (int)p.offsets[i];
         }
         s_part[tid] = local;
-        if (tid == 0) s_abort = 0;
         __syncthreads();
         DECODE_TRACE(12);
         if (wid == 0) {
@@ -253,14 +265,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         if (i1 == n && i0 < n) s_P[n] = run;
         if (n == 0 && tid == 0) s_P[0] = 0;
-        if (tid == 0) {
-            for (int s = 0; s < kStages; ++s) {
-                mbar_init(smem_u32(&s_bar[s]), 1);             // full: the producer's expect_tx arrival
-                mbar_init(smem_u32(&s_bar[kStages + s]), NCW);  // empty: one arrival per consumer warp
-            }
-            mbar_init(smem_u32(&s_bar[2 * kStages]), 1);        // partials staged for the final merge
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
         __syncthreads();
     }
     DECODE_TRACE(13);
@@ -743,8 +747,17 @@ int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st
     const int ctas = sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas;
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, HKV, G_HI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            C::SMEM_BYTES));
-    decode_kernel<D, HKV, G_HI><<<ctas, C::THREADS, C::SMEM_BYTES, st>>>(tm_k, tm_v, p);
-    AIRCACHE_LAUNCH_CHECK();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    AIRCACHE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel<D, HKV, G_HI>, tm_k, tm_v, p));
     return AIRCACHE_OK;
 }
 
