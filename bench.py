@@ -47,7 +47,7 @@ L2_BYTES = 126 * 2 ** 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from the ncu capture summarised
 # in profiles/; valid only for the kernel source it was taken on (sha1 of csrc/decode.cu, first 12 hex).
-NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "", "bytes_per_launch": None}
+NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "12524555492d", "bytes_per_launch": 49458000}
 
 
 def parse_args():
@@ -63,7 +63,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--extra", default="c4", help="comma list of further workloads measured briefly at N = 1 "
-                                                  "(decode and compaction rooflines); empty string to skip")
+                                                  "(decode and compaction rooflines); \"none\" to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -350,7 +350,7 @@ def run_cuda(args):
 
     # The default workload moves 49 MB per decode launch, about 7.6 us of HBM time: launch, prologue and the
     # split-K merge weigh as much as the stream.  The same kernels on the HBM-bound configurations:
-    if rank == 0 and world == 1 and args.extra:
+    if rank == 0 and world == 1 and args.extra not in ("", "none"):
         extra = {}
         for spec in args.extra.split(","):
             w2 = pick_workload(spec, None)
