@@ -374,10 +374,10 @@ def test_config2_full_size(oracle, ratio):
         assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
 
 
-@pytest.mark.parametrize("cfg,batch,seqs", [("c3", 32, (0, 31)), ("c4", 4, (1,))])
+@pytest.mark.parametrize("cfg,batch,seqs", [("c3", 32, (0, 31)), ("c4", 4, (1,)), ("c5", 8, (5,))])
 def test_batched_configs_sampled_sequences(oracle, cfg, batch, seqs):
-    """Batched 7B-shaped configurations at full batch on the GPU; the oracle runs whole sequences sampled
-    from the batch (every stage is independent per sequence, so a sequence's regions compare one to one)."""
+    """Batched configurations (7B shapes, and the 72B-shaped long-context one at its full 80 layers x 8
+    sequences) at full batch on the GPU; the oracle runs whole sequences sampled from the batch (every stage is independent per sequence, so a sequence's regions compare one to one)."""
     from workloads import full_cache, window_queries
     wl = CONFIGS[cfg].with_(batch=batch)
     gp = GpuPath(wl, device=DEV)
