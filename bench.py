@@ -58,6 +58,7 @@ def parse_args():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", help="c1 | c2 | c3[:batch] | c4 | c5")
     ap.add_argument("--ratio", type=float, default=None)
+    ap.add_argument("--alpha", type=float, default=None, help="relevance threshold of Eq. 5 (default 0.9; 0 = dense window)")
     ap.add_argument("--rotate", type=int, default=0, help="resident requests (0 = enough to exceed 2x L2)")
     ap.add_argument("--decode-steps", type=int, default=0, help="decode rounds per step (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
@@ -68,7 +69,7 @@ def parse_args():
     return ap.parse_args()
 
 
-def pick_workload(spec: str, ratio):
+def pick_workload(spec: str, ratio, alpha=None):
     from workloads import CONFIGS
     name, _, arg = spec.partition(":")
     wl = CONFIGS[name]
@@ -76,6 +77,8 @@ def pick_workload(spec: str, ratio):
         wl = wl.with_(batch=int(arg))
     if ratio is not None:
         wl = wl.with_(ratio=ratio)
+    if alpha is not None:
+        wl = wl.with_(alpha=alpha)
     return wl
 
 
@@ -308,7 +311,7 @@ def run_cuda(args):
     torch.cuda.set_device(dev)
     ac.lib()  # fail loudly if the library is missing
 
-    wl = pick_workload(args.workload, args.ratio)
+    wl = pick_workload(args.workload, args.ratio, args.alpha)
     n_dec = args.decode_steps or wl.steps
     sh = shape_of(ac, wl)
     rotate, cache_bytes = default_rotate(ac, wl)
@@ -345,6 +348,8 @@ def run_cuda(args):
     }
     if rank == 0 and not args.no_e2e:
         result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 5))
+    if rank == 0 and world == 1 and args.extra not in ("", "none"):
+        result["score_dense_window"] = dense_window_score(wl, reqs[0])
     del reqs
     torch.cuda.empty_cache()
 
@@ -374,6 +379,26 @@ def run_cuda(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(result))
+
+
+def dense_window_score(wl, s, reps=10):
+    """aircache_score with alpha = 0 (every window query is an elite row: Eq. 7 becomes a dense
+    [G*W x N_v] contraction per KV head, computed by the tcgen05 kernels), timed on one resident request."""
+    for _ in range(3):
+        s.score(s.qw, alpha=0.0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        s.score(s.qw, alpha=0.0)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    rows = wl.group * wl.window
+    flops = 2 * 2.0 * rows * wl.n_visual * wl.head_dim * wl.n_kv_heads * wl.n_layers * wl.batch   # two passes
+    return {"alpha": 0.0, "rows_per_kv_group": rows, "us_per_request": us, "tflops": flops / (us * 1e-6) / 1e12,
+            "key_bytes": wl.n_visual * wl.n_kv_heads * wl.head_dim * 2 * wl.n_layers * wl.batch,
+            "note": "both passes of Eq. 7 on tcgen05; FLOPs count the unpadded rows, keys are read once per pass"}
 
 
 def describe(wl):

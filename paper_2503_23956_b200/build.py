@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libaircache.so")
 SOURCES = ["api.cu", "score.cu", "budget.cu", "compact.cu", "decode.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(os.path.dirname(PKG), "include", "aircache.h")]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "ptx.cuh"), os.path.join(os.path.dirname(PKG), "include", "aircache.h")]
 
 
 def _nvcc() -> str:

@@ -21,6 +21,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace aircache {
 
@@ -45,6 +46,9 @@ struct ScoreParams {
     int keep_all;
     // one stats launch handles the KV groups with rows_lo < elite rows <= rows_hi
     int rows_lo, rows_hi;
+    // dense (tcgen05) path: position of the token / head / sequence / layer coordinate in the key tensor map
+    int pos_token, pos_head, pos_batch, pos_layer;
+    uint32_t *status;
 };
 
 constexpr float kNegBig = -1.0e30f;
@@ -394,6 +398,319 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Dense window (alpha = 0: every one of the G*W window queries is an elite row, Eq. 7 is a dense
+// [G*W x N_v] contraction per KV head).  Same two passes on the 5th-generation tensor cores:
+//   * key tiles of 128 tokens come in by TMA (5-D tensor map over the caller's strided cache, 128-byte
+//     swizzle), query blocks of 128 rows are written into the same K-major swizzled layout by the threads;
+//   * one thread issues tcgen05.mma (M = 128, N = 128, K = 16 per instruction), the accumulator lives in
+//     tensor memory and is read back with tcgen05.ld, one accumulator row per thread;
+//   * pass one puts the query rows on M, so a thread owns one softmax row and keeps its running (max, sum)
+//     in two registers; pass two swaps the operands (the same two shared-memory tiles), so a thread owns one
+//     key and sums the weighted probabilities of all rows - neither pass needs a cross-lane reduction.
+// Every mbarrier wait is bounded (status word + CTA-wide abort flag, as in the decode kernel).
+// ---------------------------------------------------------------------------------------------
+template <int D>
+struct DenseCfg {
+    static constexpr int KSUB = D / 64;             // 64-channel sub-tiles: rows of 128 bytes
+    static constexpr int SUB_BYTES = 128 * 128;     // 128 rows
+    static constexpr int TILE_BYTES = KSUB * SUB_BYTES;
+    static constexpr int NST = 2;                   // key tiles in flight (two CTAs share an SM)
+    static constexpr int SMEM_STATS = 1024 + (NST + 1) * TILE_BYTES + 256;
+    static constexpr int KT = 4;                    // key tiles per CTA of the importance pass
+    static constexpr int SMEM_IMP = 1024 + (NST + 1) * TILE_BYTES + 128 * 8 + 256;
+};
+
+// 128 query rows (row0 .. row0+127 of the group's table, zero beyond) into the swizzled K-major layout.
+// 128 threads: thread t copies 16-byte chunk t % (D/8) of rows t / (D/8) + k * (1024 / D); all table entries are
+// fetched first, then all query chunks, so the copy costs two memory round trips.
+template <int D>
+__device__ __forceinline__ void stage_queries_sw128(uint8_t *s_q, const ScoreParams &p, int grp, int lb, int g,
+                                                    int row0, int n_rows) {
+    constexpr int SUB = DenseCfg<D>::SUB_BYTES;
+    constexpr int CPR = D / 8;            // 16-byte chunks per row
+    constexpr int RPI = 128 / CPR;        // rows covered by the CTA per step
+    constexpr int STEPS = 128 / RPI;
+    const int32_t *info = p.row_info + (int64_t)grp * p.cap;
+    const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * D;
+    const int c16 = threadIdx.x % CPR, r0 = threadIdx.x / CPR;
+    int in[STEPS];
+#pragma unroll
+    for (int k = 0; k < STEPS; ++k) {
+        const int r = row0 + r0 + k * RPI;
+        in[k] = r < n_rows ? __ldg(info + r) : -1;
+    }
+    uint4 v[STEPS];
+#pragma unroll
+    for (int k = 0; k < STEPS; ++k) {
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (in[k] >= 0) {
+            const int hl = in[k] >> 8, w = in[k] & 255;
+            v[k] = __ldg(reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D) + c16);
+        }
+    }
+    const int sub = c16 >> 3, cc = c16 & 7;
+#pragma unroll
+    for (int k = 0; k < STEPS; ++k) {
+        const int r = r0 + k * RPI;
+        *reinterpret_cast<uint4 *>(s_q + sub * SUB + r * 128 + ((cc ^ (r & 7)) << 4)) = v[k];
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes, read by the tensor core
+}
+
+// acc[128 x 128] = A[128 x D] * B[128 x D]^T, both tiles K-major swizzled at a_base / b_base.
+template <int D>
+__device__ __forceinline__ void issue_tile_mma(uint32_t tmem_d, uint32_t a_base, uint32_t b_base) {
+    constexpr int SUB = DenseCfg<D>::SUB_BYTES;
+    const uint32_t idesc = umma_idesc_bf16(128, 128);
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t off = (kk >> 2) * SUB + (kk & 3) * 32;
+        umma_bf16(tmem_d, umma_desc_sw128(a_base + off), umma_desc_sw128(b_base + off), idesc, kk > 0 ? 1u : 0u);
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void load_key_tile(uint32_t dst, const CUtensorMap *tm, const ScoreParams &p, int key,
+                                              int g, int b, int l, uint32_t bar) {
+    int c[5] = {0, 0, 0, 0, 0};
+    c[p.pos_token] = key; c[p.pos_head] = g; c[p.pos_batch] = b; c[p.pos_layer] = l;
+    mbar_expect_tx(bar, DenseCfg<D>::TILE_BYTES);
+#pragma unroll
+    for (int sub = 0; sub < DenseCfg<D>::KSUB; ++sub)
+        tma_load_5d(dst + sub * DenseCfg<D>::SUB_BYTES, tm, sub * 64, c[1], c[2], c[3], c[4], bar);
+}
+
+// Pass one, dense.  grid = (chunks, L*B*Hkv), 128 threads.
+template <int D>
+__global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+    using C = DenseCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *s_k = smem;                             // NST key tiles
+    uint8_t *s_q = smem + C::NST * C::TILE_BYTES;    // one query block
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES);   // full[NST], done
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort, s_is_last;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int grp = blockIdx.y;
+    const int g = grp % p.Hkv, lb = grp / p.Hkv;
+    const int l = lb / p.B, b = lb % p.B;
+    const int chunk = blockIdx.x;
+    const int key0 = chunk * p.chunk_keys, key1 = min(p.Nv, key0 + p.chunk_keys);
+    const int n_tiles = key1 > key0 ? (key1 - key0 + 127) / 128 : 0;
+    const int n_rows = p.row_count[grp];
+    float2 *out = p.chunk_stats + ((int64_t)grp * p.chunks + chunk) * p.cap;
+
+    if (tid == 0) {
+        for (int i = 0; i <= C::NST; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_abort = 0;
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const uint32_t done_bar = smem_u32(&s_bar[C::NST]);
+    uint32_t n_loaded = 0, n_done = 0;   // running counts: they give stage and mbarrier parity
+    bool ok = true;
+
+    for (int row0 = 0; row0 < n_rows && ok; row0 += 128) {
+        __syncthreads();
+        stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
+        __syncthreads();
+        float m = kNegBig, z = 0.f;
+        const uint32_t first = n_loaded;
+        if (tid == 0)
+            for (int i = 0; i < min(C::NST, n_tiles); ++i, ++n_loaded)
+                load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p, key0 + i * 128, g, b, l,
+                                 smem_u32(&s_bar[n_loaded % C::NST]));
+        for (int t = 0; t < n_tiles; ++t) {
+            const uint32_t it = first + t, st = it % C::NST;
+            if (tid == 0) {
+                ok = mbar_wait(smem_u32(&s_bar[st]), (it / C::NST) & 1, &s_abort, p.status, 4);
+                if (ok) {
+                    tc_fence_after();
+                    // rows on M: acc[row][key] = Q_blk * K_tile^T
+                    issue_tile_mma<D>(tmem, smem_u32(s_q), smem_u32(s_k + st * C::TILE_BYTES));
+                    umma_commit(done_bar);
+                }
+            }
+            ok = mbar_wait(done_bar, n_done & 1, &s_abort, p.status, 5);
+            ++n_done;
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int cc = 0; cc < 4; ++cc) {
+                float v[32];
+                tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + cc * 32, v);
+                const int kbase = key0 + t * 128 + cc * 32;
+                float mx = kNegBig;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    v[j] = kbase + j < key1 ? v[j] * p.sl2 : kNegBig;
+                    mx = fmaxf(mx, v[j]);
+                }
+                const float mn = fmaxf(m, mx);
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) sum += kbase + j < key1 ? fast_exp2(v[j] - mn) : 0.f;
+                z = z * fast_exp2(m - mn) + sum;
+                m = mn;
+            }
+            tc_fence_before();
+            __syncthreads();   // the accumulator and the key stage are free again
+            if (tid == 0 && t + C::NST < n_tiles) {
+                load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p,
+                                 key0 + (t + C::NST) * 128, g, b, l, smem_u32(&s_bar[n_loaded % C::NST]));
+                ++n_loaded;
+            }
+        }
+        n_loaded = first + n_tiles;   // every thread tracks the count thread 0 advanced
+        if (ok && row0 + tid < n_rows) __stcg(out + row0 + tid, make_float2(m, z));
+    }
+    ok = !s_abort;
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (!ok) return;
+
+    // last CTA of the group: merge text and chunk statistics (same scheme as stats_kernel)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        s_is_last = atomicAdd(p.group_ticket + grp, 1u) == (unsigned)p.chunks - 1;
+        if (s_is_last) __threadfence();
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    for (int r = warp; r < n_rows; r += 4) {
+        float mm = kNegBig, zz = 0.f;
+        if (lane == 0) {
+            const float2 tx = p.row_text[(int64_t)grp * p.cap + r];
+            mm = tx.x; zz = tx.y;
+        }
+        for (int c = lane; c < p.chunks; c += 32) {
+            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)grp * p.chunks + c) * p.cap + r);
+            merge_stats(mm, zz, cs.x, cs.y);
+        }
+#pragma unroll
+        for (int sh = 1; sh < 32; sh <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mm, sh);
+            const float z2 = __shfl_xor_sync(0xffffffffu, zz, sh);
+            merge_stats(mm, zz, m2, z2);
+        }
+        if (lane == 0) p.row_final[(int64_t)grp * p.cap + r] = make_float2(mm, p.row_coef[(int64_t)grp * p.cap + r] / zz);
+    }
+}
+
+// Pass two, dense.  grid = (ceil(Nv / (128 * KT)), L*B), 128 threads; a CTA owns KT key tiles and thread i the
+// keys 128 * tile + i of them.  Per KV head and block of 128 query rows the block is staged once and the
+// CTA's key tiles stream through a ring of NST stages.
+template <int D>
+__global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+    using C = DenseCfg<D>;
+    constexpr int KT = C::KT;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *s_k = smem;                             // NST key tiles
+    uint8_t *s_q = smem + C::NST * C::TILE_BYTES;    // one query block
+    float2 *s_stat = reinterpret_cast<float2 *>(smem + (C::NST + 1) * C::TILE_BYTES);   // (max, weight / normaliser)
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES + 128 * 8);   // full[NST], done
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int lb = blockIdx.y;
+    const int l = lb / p.B, b = lb % p.B;
+    const int key0 = blockIdx.x * 128 * KT;
+    const int n_tiles = min(KT, (p.Nv - key0 + 127) / 128);
+
+    if (tid == 0) {
+        for (int i = 0; i <= C::NST; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_abort = 0;
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const uint32_t done_bar = smem_u32(&s_bar[C::NST]);
+    uint32_t n_loaded = 0, n_done = 0;
+    bool ok = true;
+    float imp[KT];
+#pragma unroll
+    for (int t = 0; t < KT; ++t) imp[t] = 0.f;
+
+    for (int g = 0; g < p.Hkv && ok; ++g) {
+        const int grp = lb * p.Hkv + g;
+        const int n_rows = p.row_count[grp];
+        for (int row0 = 0; row0 < n_rows && ok; row0 += 128) {
+            const uint32_t first = n_loaded;
+            if (tid == 0)   // the ring is empty here: every tile of the previous block was consumed
+                for (int i = 0; i < min(C::NST, n_tiles); ++i, ++n_loaded)
+                    load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p, key0 + i * 128, g, b,
+                                     l, smem_u32(&s_bar[n_loaded % C::NST]));
+            stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
+            s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
+            __syncthreads();
+            const int cols = min(128, n_rows - row0);
+#pragma unroll
+            for (int t = 0; t < KT; ++t) {
+                if (t >= n_tiles) break;
+                const uint32_t it = first + t, st = it % C::NST;
+                if (tid == 0) {
+                    ok = mbar_wait(smem_u32(&s_bar[st]), (it / C::NST) & 1, &s_abort, p.status, 6);
+                    if (ok) {
+                        tc_fence_after();
+                        // keys on M: acc[key][row] = K_tile * Q_blk^T
+                        issue_tile_mma<D>(tmem, smem_u32(s_k + st * C::TILE_BYTES), smem_u32(s_q));
+                        umma_commit(done_bar);
+                    }
+                }
+                ok = mbar_wait(done_bar, n_done & 1, &s_abort, p.status, 7);
+                ++n_done;
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int cc = 0; cc < 4; ++cc) {
+                    if (cc * 32 >= cols) break;
+                    float v[32];
+                    tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + cc * 32, v);
+                    float acc = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float2 sj = s_stat[cc * 32 + j];
+                        acc += fast_exp2(v[j] * p.sl2 - sj.x) * sj.y;
+                    }
+                    imp[t] += acc;
+                }
+                tc_fence_before();
+                __syncthreads();   // accumulator and key stage are free again
+                if (tid == 0 && t + C::NST < n_tiles) {
+                    load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p,
+                                     key0 + (t + C::NST) * 128, g, b, l, smem_u32(&s_bar[n_loaded % C::NST]));
+                    ++n_loaded;
+                }
+            }
+            n_loaded = first + n_tiles;
+        }
+    }
+    ok = !s_abort;
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (!ok) return;
+#pragma unroll
+    for (int t = 0; t < KT; ++t) {
+        const int key = key0 + t * 128 + tid;
+        if (t < n_tiles && key < p.Nv) p.scores[(int64_t)lb * p.Nv + key] = imp[t];
+    }
+}
+
 template <int D, int NT>
 int launch_stats(ScoreParams p, int rows_lo, int rows_hi, cudaStream_t st) {
     p.rows_lo = rows_lo; p.rows_hi = rows_hi;
@@ -432,6 +749,52 @@ int launch_passes_d(const ScoreParams &p, cudaStream_t st) {
     return nt_max <= 4 ? launch_importance<D, 4>(p, st) : launch_importance<D, 8>(p, st);
 }
 
+// 5-D tensor map over the caller's key cache: channels innermost, then token / head / sequence / layer in
+// the order of their strides (smallest first); one box = 64 channels x 128 tokens.
+int make_key_map(CUtensorMap *tm, ScoreParams &p, const aircache_shape_t *s, const aircache_full_t *f) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return AIRCACHE_ERR_CUDA;
+    struct Dim { int64_t size, stride; int which; };
+    Dim dims[4] = {{(int64_t)s->n_visual + s->n_text, f->stride_token, 0}, {s->n_kv_heads, f->stride_head, 1},
+                   {s->batch, f->stride_batch, 2}, {s->n_layers, f->stride_layer, 3}};
+    for (int i = 0; i < 4; ++i)
+        for (int j = i + 1; j < 4; ++j)
+            if (dims[j].stride < dims[i].stride || (dims[j].stride == dims[i].stride && dims[j].size < dims[i].size)) {
+                const Dim t = dims[i]; dims[i] = dims[j]; dims[j] = t;
+            }
+    cuuint64_t gdim[5] = {(cuuint64_t)s->head_dim, 1, 1, 1, 1};
+    cuuint64_t gstr[4] = {0, 0, 0, 0};
+    cuuint32_t box[5] = {64, 1, 1, 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    int pos[4] = {0, 0, 0, 0};
+    for (int i = 0; i < 4; ++i) {
+        gdim[i + 1] = (cuuint64_t)dims[i].size;
+        // a dimension of extent 1 never moves; give it the smallest stride the encoder accepts
+        gstr[i] = (cuuint64_t)(dims[i].stride > 0 ? dims[i].stride : s->head_dim) * 2;
+        pos[dims[i].which] = i + 1;
+        if (dims[i].which == 0) box[i + 1] = 128;
+    }
+    p.pos_token = pos[0]; p.pos_head = pos[1]; p.pos_batch = pos[2]; p.pos_layer = pos[3];
+    const CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(f->k), gdim, gstr, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? AIRCACHE_OK : AIRCACHE_ERR_CUDA;
+}
+
+template <int D>
+int launch_dense(ScoreParams &p, const CUtensorMap &tm, cudaStream_t st) {
+    using C = DenseCfg<D>;
+    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_STATS));
+    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_importance_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           C::SMEM_IMP));
+    dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.L * p.B * p.Hkv)), 128, C::SMEM_STATS, st>>>(tm, p);
+    AIRCACHE_LAUNCH_CHECK();
+    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)((int64_t)p.L * p.B)), 128,
+                                 C::SMEM_IMP, st>>>(tm, p);
+    AIRCACHE_LAUNCH_CHECK();
+    return AIRCACHE_OK;
+}
+
 }  // namespace
 
 int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void *q_window, float alpha,
@@ -460,12 +823,23 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.keep_all = alpha <= 0.0f;
     p.ln_alpha = p.keep_all ? 0.0f : (float)log((double)alpha);
     p.rows_lo = 0; p.rows_hi = 1 << 30;
+    p.pos_token = p.pos_head = p.pos_batch = p.pos_layer = 0;
+    p.status = ws_ptr<uint32_t>(ws, w.status);
 
     const int64_t groups = (int64_t)p.L * p.B * p.Hkv;
     const size_t elite_smem = (size_t)(p.W + p.G) * (p.d + 8) * 2;
     if (s->head_dim == 64) elite_kernel<64><<<(unsigned)groups, 128, elite_smem, st>>>(p);
     else elite_kernel<128><<<(unsigned)groups, 128, elite_smem, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
+    // alpha = 0 keeps all G*W window queries: the dense contraction goes to tcgen05 (if a tensor map over the
+    // caller's strides can be made; otherwise the mma.sync passes handle it as well)
+#ifndef AIRCACHE_NO_DENSE
+    if (p.keep_all && p.G * p.W >= 32) {
+        CUtensorMap tm;
+        if (make_key_map(&tm, p, s, f) == AIRCACHE_OK)
+            return s->head_dim == 64 ? launch_dense<64>(p, tm, st) : launch_dense<128>(p, tm, st);
+    }
+#endif
     return s->head_dim == 64 ? launch_passes_d<64>(p, st) : launch_passes_d<128>(p, st);
 }
 
