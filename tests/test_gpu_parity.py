@@ -102,6 +102,31 @@ def test_score_parity(oracle, case, alpha):
     assert err <= TOL, err
 
 
+@pytest.mark.parametrize("alpha", [0.9, 0.0])
+@pytest.mark.parametrize("layout", ["head_major", "layer_innermost"])
+def test_score_parity_other_cache_layouts(oracle, alpha, layout):
+    """The same scores from a head-major cache [L,B,Hkv,N,d] and from one whose layer stride is the smallest
+    ([B,Hkv,N,L,d] storage): the kernels (and, for alpha = 0, the tensor map of the dense path) only see strides."""
+    wl = CASES["s7b"]
+    ref = oracle_path(oracle, wl, alpha=alpha)
+    kl, vl = logical(ref["k"]), logical(ref["v"])                      # logical [L,B,Hkv,N,d]
+    if layout == "head_major":
+        kd, vd = kl.contiguous().to(DEV), vl.contiguous().to(DEV)
+    else:
+        kd = kl.permute(1, 2, 3, 0, 4).contiguous().to(DEV).permute(3, 0, 1, 2, 4)
+        vd = vl.permute(1, 2, 3, 0, 4).contiguous().to(DEV).permute(3, 0, 1, 2, 4)
+    gp = GpuPath(wl, ratio=ref["ratio"], device=DEV)
+    gp.set_full(kd, vd)
+    gp.score(ref["qw"].to(DEV), alpha=alpha)
+    assert gp.status() == 0
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"])
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+    gp.budget()
+    gp.compact()
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+    compare_cache(gp, ref["compact"])
+
+
 @pytest.mark.parametrize("case", ["c1", "s7b", "mha64"])
 @pytest.mark.parametrize("mode", [0, 1, 2, 3])
 @pytest.mark.parametrize("ratio", [0.1, 0.83])
