@@ -63,6 +63,7 @@ struct DecodeParams {
     float *partials;         // [2 * CTAs][Hq * (D + 2)]
     uint32_t *status;
     int n_regions, Hq, G;
+    int hs;                  // head-split mode: KV heads per region (items are (region, head) pairs); else 1
     float sl2;               // scale * log2(e)
 };
 
@@ -89,10 +90,10 @@ __device__ __forceinline__ float exp2_or_zero(float m, float m_new) {
     return m == -INFINITY ? 0.f : fast_exp2(m - m_new);
 }
 
-template <int D, int HKV, bool G_HI>
+template <int D, int HKV, bool G_HI, bool HS>
 struct DecodeCfg {
     static constexpr int NROW = G_HI ? 2 : 1;        // accumulator row groups in use (heads 0-7, heads 8-15)
-    static constexpr int KSPLIT = (8 / HKV) > 4 ? 4 : (8 / HKV);
+    static constexpr int KSPLIT = HS ? 8 : ((8 / HKV) > 4 ? 4 : (8 / HKV));
     static constexpr int CH = 16 * KSPLIT;           // rows per unit
     static constexpr int NCW = HKV * KSPLIT;         // consumer warps
     static constexpr int THREADS = (NCW + 1) * 32;
@@ -100,9 +101,9 @@ struct DecodeCfg {
     static constexpr int SUBTILE = CH * 128;         // bytes of one (head, half) box
     static constexpr int KV_BYTES = HKV * HALVES * SUBTILE;
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
-    // merge buffer: one slot per consumer warp with ks > 0
     static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 2));
-    static constexpr int MERGE_BYTES = HKV * (KSPLIT - 1) * MERGE_FLOATS_PER_WARP * 4;
+    static constexpr int MERGE_SLOTS = KSPLIT / 2;     // tree merge: the upper half of the warps hands over to the lower
+    static constexpr int MERGE_BYTES = HKV * MERGE_SLOTS * MERGE_FLOATS_PER_WARP * 4;
     // the prologue's scan scratch lives in the same bytes as the merge buffer (used before the first flush)
     static constexpr int SCAN_BYTES = THREADS * 4;
     static constexpr int MERGE_STAGE_BYTES = 16384;            // weights [partials][Hq] of the final merge
@@ -138,10 +139,10 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
     return lo;
 }
 
-template <int D, int HKV, bool G_HI>
-__global__ void __launch_bounds__(DecodeCfg<D, HKV, G_HI>::THREADS, 1)
+template <int D, int HKV, bool G_HI, bool HS>
+__global__ void __launch_bounds__(DecodeCfg<D, HKV, G_HI, HS>::THREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, DecodeParams p) {
-    using C = DecodeCfg<D, HKV, G_HI>;
+    using C = DecodeCfg<D, HKV, G_HI, HS>;
     constexpr int KSPLIT = C::KSPLIT, CH = C::CH, NCW = C::NCW, NROW = C::NROW, kStages = C::NSTAGE;
 
     DECODE_TRACE(0);
@@ -160,7 +161,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __shared__ int s_aligned;
 
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
-    const int n = p.n_regions;
+    const int n = p.n_regions;   // items: regions, or (region, KV head) pairs in head-split mode
+    const int hs = HS ? p.hs : 1;
     const int n_ctas = (int)gridDim.x;
     // Programmatic dependent launch: the next kernel in the stream may be scheduled as soon as SMs free up,
     // and this one does everything that reads no global memory before it waits for its predecessor.
@@ -186,8 +188,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
         int local = 0;
         for (int i = i0; i < i1; ++i) {
-            local += (max(p.lens[i], 0) + CH - 1) / CH;
-            s_off[i] = (int)p.offsets[i];
+            local += (max(p.lens[i / hs], 0) + CH - 1) / CH;
+            s_off[i] = (int)p.offsets[i / hs];
         }
         s_part[tid] = local;
         __syncthreads();
@@ -216,7 +218,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         int run = s_part[tid];
         for (int i = i0; i < i1; ++i) {
             s_P[i] = run;
-            run += (max(p.lens[i], 0) + CH - 1) / CH;
+            run += (max(p.lens[i / hs], 0) + CH - 1) / CH;
         }
         if (i1 == n && i0 < n) s_P[n] = run;
         if (n == 0 && tid == 0) s_P[0] = 0;
@@ -230,23 +232,49 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // Region-aligned mode (few regions, each cut into pieces of at most upc units, if that needs no more
     // CTAs than there are): every CTA works on one region only, so it reloads no query and flushes once.
     if (wid == 0) {
-        // pieces per region and their exclusive prefix, 32 regions per round (rolled: this runs once)
-        const bool few = n <= n_ctas;
+        // Aligned pieces of at most upc_a units: upc_a is the smallest of upc, upc + 1, upc + 2 for which the
+        // pieces need no more CTAs than the grid has (two more units on the longest CTA cost less than a
+        // second flush and merge).  All items of a region have the same unit count, so the sums run over
+        // regions; the three candidates are evaluated together.  Rolled loops: this runs once.
+        const bool few = n <= n_ctas && total > 0;
+        const int nr = n / hs;
+        int sum0 = 0, sum1 = 0, sum2 = 0;
+#pragma unroll 1
+        for (int r = lane; few && r < nr; r += 32) {
+            const int u = s_P[r * hs + 1] - s_P[r * hs];
+            sum0 += small_div(u + upc - 1, upc);
+            sum1 += small_div(u + upc, upc + 1);
+            sum2 += small_div(u + upc + 1, upc + 2);
+        }
+#pragma unroll
+        for (int sh = 16; sh > 0; sh >>= 1) {
+            sum0 += __shfl_xor_sync(0xffffffffu, sum0, sh);
+            sum1 += __shfl_xor_sync(0xffffffffu, sum1, sh);
+            sum2 += __shfl_xor_sync(0xffffffffu, sum2, sh);
+        }
+        const int lim = n_ctas / hs;   // the sums count pieces per head
+        const bool found = few && (sum0 <= lim || sum1 <= lim || sum2 <= lim);
+        const int upc_a = sum0 <= lim ? upc : (sum1 <= lim ? upc + 1 : upc + 2);
         int carry = 0;
 #pragma unroll 1
-        for (int base = 0; few && base <= n; base += 32) {
+        for (int base = 0; found && base <= nr; base += 32) {
             const int r = base + lane;
-            const int v = r < n ? small_div(s_P[r + 1] - s_P[r] + upc - 1, upc) : 0;
+            const int v = r < nr ? small_div(s_P[r * hs + 1] - s_P[r * hs] + upc_a - 1, upc_a) : 0;
             int incl = v;
 #pragma unroll
             for (int sh = 1; sh < 32; sh <<= 1) {
                 const int o = __shfl_up_sync(0xffffffffu, incl, sh);
                 if (lane >= sh) incl += o;
             }
-            if (r <= n) s_Q[r] = carry + incl - v;
+            if (r < nr) {
+#pragma unroll 1
+                for (int h = 0; h < hs; ++h) s_Q[r * hs + h] = (carry + incl - v) * hs + h * v;
+            } else if (r == nr) {
+                s_Q[n] = (carry + incl - v) * hs;
+            }
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
-        if (lane == 0) s_aligned = (few && total > 0 && carry <= n_ctas) ? 1 : 0;
+        if (lane == 0) s_aligned = found ? 1 : 0;
     }
     __syncthreads();
     DECODE_TRACE(14);
@@ -303,8 +331,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
                     for (int hf = 0; hf < C::HALVES; ++hf) {
                         const uint32_t off = (g * C::HALVES + hf) * C::SUBTILE;
-                        tma_load_3d(dst + off, &tm_k, hf * 64, g, row0, full);
-                        tma_load_3d(dst + C::KV_BYTES + off, &tm_v, hf * 64, g, row0, full);
+                        const int head = HS ? r % hs : g;
+                        tma_load_3d(dst + off, &tm_k, hf * 64, head, row0, full);
+                        tma_load_3d(dst + C::KV_BYTES + off, &tm_v, hf * 64, head, row0, full);
                     }
                 }
             }
@@ -353,10 +382,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
             l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
         }
-        if (KSPLIT > 1) {
-            constexpr int REGS = NROW * (D / 4 + 2);
-            if (ks > 0) {
-                float *dst = s_merge + (size_t)(g * (KSPLIT - 1) + ks - 1) * C::MERGE_FLOATS_PER_WARP + lane;
+        // the KSPLIT warps of a KV head merge their states pairwise: in every round the upper half of the
+        // remaining warps hands its (max, sum, accumulator) to the lower half through shared memory
+#pragma unroll
+        for (int half = KSPLIT / 2; half >= 1; half >>= 1) {
+            if (ks >= half && ks < 2 * half) {
+                float *dst = s_merge + (size_t)(g * C::MERGE_SLOTS + ks - half) * C::MERGE_FLOATS_PER_WARP + lane;
                 int c = 0;
 #pragma unroll
                 for (int i = 0; i < NROW; ++i) {
@@ -368,26 +399,23 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         dst[32 * c++] = oacc[nd][2 * i + 1];
                     }
                 }
-                (void)REGS;
             }
             consumer_bar(NCW * 32);
-            if (ks == 0) {
-                for (int o = 0; o < KSPLIT - 1; ++o) {
-                    const float *src = s_merge + (size_t)(g * (KSPLIT - 1) + o) * C::MERGE_FLOATS_PER_WARP + lane;
-                    int c = 0;
+            if (ks < half) {
+                const float *src = s_merge + (size_t)(g * C::MERGE_SLOTS + ks) * C::MERGE_FLOATS_PER_WARP + lane;
+                int c = 0;
 #pragma unroll
-                    for (int i = 0; i < NROW; ++i) {
-                        const float m2 = src[32 * c++];
-                        const float l2 = src[32 * c++];
-                        const float mn = fmaxf(m_run[i], m2);
-                        const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
-                        l_run[i] = l_run[i] * a + l2 * b;
-                        m_run[i] = mn;
+                for (int i = 0; i < NROW; ++i) {
+                    const float m2 = src[32 * c++];
+                    const float l2 = src[32 * c++];
+                    const float mn = fmaxf(m_run[i], m2);
+                    const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
+                    l_run[i] = l_run[i] * a + l2 * b;
+                    m_run[i] = mn;
 #pragma unroll
-                        for (int nd = 0; nd < D / 8; ++nd) {
-                            oacc[nd][2 * i] = oacc[nd][2 * i] * a + src[32 * c++] * b;
-                            oacc[nd][2 * i + 1] = oacc[nd][2 * i + 1] * a + src[32 * c++] * b;
-                        }
+                    for (int nd = 0; nd < D / 8; ++nd) {
+                        oacc[nd][2 * i] = oacc[nd][2 * i] * a + src[32 * c++] * b;
+                        oacc[nd][2 * i + 1] = oacc[nd][2 * i + 1] * a + src[32 * c++] * b;
                     }
                 }
             }
@@ -536,7 +564,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     int r = find_region(s_P, n, u0);
     int seg_start = u0;
-    int len = p.lens[r];
+    int len = p.lens[r / hs];
     load_q(r);
     int it = 0;
     bool ok = true;
@@ -548,7 +576,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             n_flush = n_flush < 2 ? n_flush + 1 : 2;
             while (u >= s_P[r + 1]) ++r;
             seg_start = u;
-            len = p.lens[r];
+            len = p.lens[r / hs];
             load_q(r);
         }
         const int s = it % kStages;
@@ -674,17 +702,17 @@ int sm_count(int *out) {
     return AIRCACHE_OK;
 }
 
-template <int D, int HKV, bool G_HI>
-int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
-    using C = DecodeCfg<D, HKV, G_HI>;
+template <int D, int HKV, bool G_HI, bool HS>
+int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, int kv_heads, cudaStream_t st) {
+    using C = DecodeCfg<D, HKV, G_HI, HS>;
     CUtensorMap tm_k, tm_v;
-    int rc = make_map(&tm_k, c->k, D, HKV, c->total_rows, C::CH);
+    int rc = make_map(&tm_k, c->k, D, kv_heads, c->total_rows, C::CH);
     if (rc) return rc;
-    if ((rc = make_map(&tm_v, c->v, D, HKV, c->total_rows, C::CH))) return rc;
+    if ((rc = make_map(&tm_v, c->v, D, kv_heads, c->total_rows, C::CH))) return rc;
     int sms = 0;
     if ((rc = sm_count(&sms))) return rc;
     const int ctas = sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas;
-    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, HKV, G_HI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, HKV, G_HI, HS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            C::SMEM_BYTES));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctas);
@@ -696,18 +724,36 @@ int launch_decode_t(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    AIRCACHE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel<D, HKV, G_HI>, tm_k, tm_v, p));
+    AIRCACHE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_kernel<D, HKV, G_HI, HS>, tm_k, tm_v, p));
     return AIRCACHE_OK;
 }
 
 template <int D, int HKV>
 int launch_decode_g(const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
-    return p.G > 8 ? launch_decode_t<D, HKV, true>(c, p, st) : launch_decode_t<D, HKV, false>(c, p, st);
+    return p.G > 8 ? launch_decode_t<D, HKV, true, false>(c, p, HKV, st)
+                   : launch_decode_t<D, HKV, false, false>(c, p, HKV, st);
 }
 
+// When there are so few regions that even (region, KV head) pairs do not outnumber the SMs, the cache is cut
+// by such pairs instead of by regions: an item is then a quarter (an eighth) of a region, most items fit one
+// CTA whole and need no split-K merge, and the partials of the rest are a head's worth.  All eight consumer
+// warps work on the item's head, 128 rows per unit.  The kernel is the one-KV-head instantiation with the
+// head taken from the item index.  With more items than SMs the by-region cut is faster (shorter units, all
+// heads of a row in one contiguous read).
 template <int D>
 int launch_decode_d(const aircache_shape_t *s, const aircache_ragged_t *c, DecodeParams &p, cudaStream_t st) {
-    switch (s->n_kv_heads) {
+    const int hkv = s->n_kv_heads;
+    int sms = 0;
+    int rc = sm_count(&sms);
+    if (rc) return rc;
+    if (hkv > 1 && p.n_regions * hkv <= (sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas)) {
+        p.hs = hkv;
+        p.n_regions *= hkv;
+        p.Hq = p.G;
+        return p.G > 8 ? launch_decode_t<D, 1, true, true>(c, p, hkv, st)
+                       : launch_decode_t<D, 1, false, true>(c, p, hkv, st);
+    }
+    switch (hkv) {
         case 1: return launch_decode_g<D, 1>(c, p, st);
         case 2: return launch_decode_g<D, 2>(c, p, st);
         case 4: return launch_decode_g<D, 4>(c, p, st);
@@ -733,6 +779,7 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.Hq = s->n_q_heads;
     p.G = s->n_q_heads / s->n_kv_heads;
     p.sl2 = s->scale * kLog2e;
+    p.hs = 1;
     return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
 }
 
@@ -784,6 +831,7 @@ int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, 
     p.Hq = s->n_q_heads;
     p.G = s->n_q_heads / s->n_kv_heads;
     p.sl2 = s->scale * kLog2e;
+    p.hs = 1;
     return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
 }
 
