@@ -47,7 +47,7 @@ L2_BYTES = 126 * 2 ** 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from the ncu capture summarised
 # in profiles/; valid only for the kernel source it was taken on (sha1 of csrc/decode.cu, first 12 hex).
-NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "12524555492d", "bytes_per_launch": 49458000}
+NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "34731875a0ef", "bytes_per_launch": 49448000}
 
 
 def parse_args():
