@@ -172,17 +172,24 @@ def decode_cu_sha1():
     return hashlib.sha1(open(p, "rb").read()).hexdigest()[:12]
 
 
-def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist):
+def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, append=False):
     """Times `steps` steps of the whole path on `rotate` resident request batches of workload `wl`.
     Returns (local numbers, the sessions) -- the caller reduces over ranks."""
     from paper_2503_23956_b200.session import Session
     from workloads import decode_queries, full_cache, window_queries
 
+    if append:
+        wl = wl.with_(slack=n_dec)   # room for one appended token per decode round (Eq. 2)
     sh = shape_of(ac, wl)
     reqs = []
     for i in range(rotate):
         w = wl.with_(seed=wl.seed + 1000 * rank + i)
         s = Session(sh, wl.ratio, wl.alpha, dev)
+        if append:
+            gen = torch.Generator(device=dev).manual_seed(wl.seed + 7 * i)
+            shape_new = (n_dec, wl.n_layers * wl.batch, wl.n_kv_heads, wl.head_dim)
+            s.k_new = torch.randn(shape_new, generator=gen, device=dev).to(torch.bfloat16)
+            s.v_new = torch.randn(shape_new, generator=gen, device=dev).to(torch.bfloat16)
         k, v = full_cache(w, "k", dev), full_cache(w, "v", dev)
         s.set_full(logical(k), logical(v))
         s.qw = window_queries(w, dev)
@@ -207,6 +214,8 @@ def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist):
     def stage_decode():
         for t in range(n_dec):
             for s in reqs:
+                if append:
+                    ac.aircache_append(s.sh, s.cache, s.k_new[t], s.v_new[t], t, stream)
                 s.decode(s.q_steps[t], out=s.out_steps[t], stream=stream)
 
     stages = [("score", stage_score), ("budget", stage_budget), ("compact", stage_compact), ("decode", stage_decode)]
@@ -372,6 +381,16 @@ def run_cuda(args):
             del q2
             torch.cuda.empty_cache()
         result["hbm_bound_workloads"] = extra
+        # Eq. 2: the same decode rounds with one new token's K/V appended to every region before each round
+        # (the cache grows over the rounds; lens change, so every launch re-derives its schedule)
+        d3 = min(n_dec, 64)
+        m3, q3 = measure(ac, wl, d3, rotate, 3, 3, not args.no_graph, dev, rank, None, append=True)
+        result["decode_with_append"] = {
+            "decode_steps": d3, "tok_s": rotate * d3 * wl.batch / (m3["stage_ms"]["decode"] * 1e-3),
+            "us_per_round": m3["stage_ms"]["decode"] * 1e3 / (rotate * d3),
+            "note": "aircache_append + aircache_decode_attn per round and request"}
+        del q3
+        torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, n_dec)
     if dist is not None:
