@@ -155,6 +155,26 @@ def test_compact_parity_on_oracle_scores_and_budgets(oracle, case, slack):
     compare_cache(gp, ref["compact"])
 
 
+@pytest.mark.parametrize("n_visual", [8195, 41000])
+def test_select_long_regions(oracle, n_visual):
+    """The shared-memory and the re-reading variants of the select (more than 8192 / 40960 visual tokens),
+    on duplicated scores."""
+    wl = small("sel_long", L=2, Hq=2, Hkv=1, d=64, B=1, Nv=n_visual, Nt=4, W=2, ratio=0.3)
+    rng = np.random.default_rng(n_visual)
+    k, v, _ = cpu_inputs(wl)
+    scores = (rng.integers(0, 1000, size=(wl.n_layers, wl.batch, wl.n_visual)) / 1024.0).astype(np.float32)
+    dm = oracle_dims(oracle, wl)
+    T = oracle.total_kept(wl.n_visual, wl.n_layers, wl.ratio)
+    budgets = np.array([[T // 3], [T - T // 3]], np.int32)
+    cp = oracle.compact(dm, 0, u16(logical(k)), u16(logical(v)), scores, budgets)
+    gp = GpuPath(wl, device=DEV)
+    gp.set_full(logical(k.to(DEV)), logical(v.to(DEV)))
+    gp.offsets.copy_(torch.from_numpy(cp["offsets"])); gp.lens.copy_(torch.from_numpy(cp["lens"]))
+    gp.compact(scores=torch.from_numpy(scores).to(DEV), budgets=torch.from_numpy(budgets).to(DEV))
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+
+
 def test_select_ties_zero_and_full_budgets(oracle):
     """Heavily duplicated scores (ties broken by the lower index), a layer that keeps nothing and one that
     keeps everything, negative zero and denormal scores; head-major source layout."""
