@@ -189,6 +189,18 @@ int aircache_decode_attn(const aircache_shape_t *shape, const aircache_ragged_t 
                          float *out, void *workspace, int64_t workspace_bytes, void *cuda_stream);
 
 /*
+ * One decode step with the KV append of Eq. 2 fused in: the new token's K and V
+ * (bf16 [L, B, Hkv, d]) are stored in the first free slack row of every region,
+ * take part in this call's attention together with the lens[r] cached rows, and
+ * lens[r] grows by one when the call completes (same result as aircache_append
+ * followed by aircache_decode_attn, in one launch).  `appended` as in
+ * aircache_append; AIRCACHE_ERR_CAPACITY on the host when the slack is used up.
+ */
+int aircache_decode_step(const aircache_shape_t *shape, aircache_ragged_t *cache, const void *q, const void *k_new,
+                         const void *v_new, int32_t appended, float *out, void *workspace, int64_t workspace_bytes,
+                         void *cuda_stream);
+
+/*
  * aircache_decode_attn for callers that cannot allocate device memory.  (An
  * addition of this library; the paper has no counterpart.)
  *

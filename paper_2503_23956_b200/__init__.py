@@ -66,6 +66,8 @@ _SIGNATURES = {
                                    C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_decode_attn": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_int64, C.c_void_p]),
+    "aircache_decode_step": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_decode_attn_static": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p,
                                               C.c_void_p]),
     "aircache_append": (C.c_int, [C.POINTER(Shape), C.POINTER(Ragged), C.c_void_p, C.c_void_p, C.c_int32,
@@ -194,6 +196,14 @@ def aircache_decode_attn(sh, cache, q, out, workspace, stream=None, check=True) 
                                     _nbytes(workspace), _stream(stream))
     if check:
         _check("aircache_decode_attn", rc)
+    return rc
+
+
+def aircache_decode_step(sh, cache, q, k_new, v_new, appended, out, workspace, stream=None, check=True) -> int:
+    rc = lib().aircache_decode_step(C.byref(sh), C.byref(cache), _ptr(q), _ptr(k_new), _ptr(v_new), appended,
+                                    _ptr(out), _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check("aircache_decode_step", rc)
     return rc
 
 

@@ -198,7 +198,21 @@ int aircache_decode_attn(const aircache_shape_t *shape, const aircache_ragged_t 
     if (!q || !out) return AIRCACHE_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return AIRCACHE_ERR_ALIGNMENT;
     if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
-    return launch_decode(shape, cache, q, out, workspace, (cudaStream_t)cuda_stream);
+    return launch_decode(shape, cache, q, nullptr, nullptr, out, workspace, (cudaStream_t)cuda_stream);
+}
+
+int aircache_decode_step(const aircache_shape_t *shape, aircache_ragged_t *cache, const void *q, const void *k_new,
+                         const void *v_new, int32_t appended, float *out, void *workspace, int64_t workspace_bytes,
+                         void *cuda_stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if ((rc = check_ragged(shape, cache, true))) return rc;
+    if (!q || !out || !k_new || !v_new || appended < 0) return AIRCACHE_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15))
+        return AIRCACHE_ERR_ALIGNMENT;
+    if (appended >= shape->slack) return AIRCACHE_ERR_CAPACITY;
+    if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
+    return launch_decode(shape, cache, q, k_new, v_new, out, workspace, (cudaStream_t)cuda_stream);
 }
 
 int aircache_decode_attn_static(const aircache_shape_t *shape, const aircache_ragged_t *cache, const void *q,

@@ -115,8 +115,8 @@ int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, 
 int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const float *scores,
                    const int32_t *budgets, double ratio, aircache_ragged_t *out, int32_t *kept_idx, void *ws,
                    cudaStream_t st);
-int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out, void *ws,
-                  cudaStream_t st);
+int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, const void *k_new,
+                  const void *v_new, float *out, void *ws, cudaStream_t st);
 int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out,
                          cudaStream_t st);
 int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,

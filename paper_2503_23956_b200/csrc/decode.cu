@@ -63,6 +63,11 @@ struct DecodeParams {
     float *partials;         // [2 * CTAs][Hq * (D + 2)]
     uint32_t *status;
     int n_regions, Hq, G;
+    const uint16_t *k_new, *v_new;   // Eq. 2: [L*B, Hkv, D] K and V of the token appended by this call, or NULL
+    uint16_t *k_cache, *v_cache;     // the ragged cache, for the appended rows
+    int32_t *lens_rw;                // lens, bumped by the last CTA when a token is appended
+    int32_t *done_ticket;            // CTAs finished (append only); zero between calls
+    int kv_heads;                    // KV heads of the cache
     int hs;                  // head-split mode: KV heads per region (items are (region, head) pairs); else 1
     float sl2;               // scale * log2(e)
 };
@@ -280,15 +285,44 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     DECODE_TRACE(14);
     const bool aligned = s_aligned != 0;
 
-    // a region without rows yields zeros
+    // an item without rows yields zeros - or, when a token is appended, that token's value (softmax over one key)
     for (int r = blockIdx.x; r < n; r += n_ctas) {
-        if (s_P[r + 1] == s_P[r])
-            for (int i = tid; i < p.Hq * D; i += C::THREADS) p.out[(int64_t)r * p.Hq * D + i] = 0.f;
+        if (s_P[r + 1] != s_P[r]) continue;
+        const int reg = r / hs;
+        for (int i = tid; i < p.Hq * D; i += C::THREADS) {
+            float v = 0.f;
+            if (p.k_new) {
+                const int kvh = HS ? r % hs : (i / D) / p.G;
+                v = bf16_to_f32(p.v_new[((int64_t)reg * p.kv_heads + kvh) * D + i % D]);
+            }
+            p.out[(int64_t)r * p.Hq * D + i] = v;
+        }
+        if (p.k_new) {
+            const int heads = HS ? 1 : p.kv_heads, h0 = HS ? r % hs : 0;
+            for (int i = tid; i < heads * D; i += C::THREADS) {
+                const int64_t src = ((int64_t)reg * p.kv_heads + h0) * D + i;
+                const int64_t dst = ((int64_t)s_off[r] * p.kv_heads + h0) * D + i;
+                p.k_cache[dst] = p.k_new[src];
+                p.v_cache[dst] = p.v_new[src];
+            }
+        }
     }
+    // Eq. 2 bookkeeping: the CTA that finishes last adds the appended token to every region's length
+    auto finish = [&](bool all_threads) {
+        if (p.k_new == nullptr) return;
+        if (tid == 0) {
+            __threadfence();
+            s_last = atomicAdd(p.done_ticket, 1) == n_ctas - 1;
+            if (s_last) *p.done_ticket = 0;
+        }
+        if (all_threads) __syncthreads(); else consumer_bar(NCW * 32);
+        if (s_last)
+            for (int i = tid; i < n / hs; i += (all_threads ? C::THREADS : NCW * 32)) p.lens_rw[i] += 1;
+    };
     int u0, u1;
     if (aligned) {
         const int c = (int)blockIdx.x;
-        if (c >= s_Q[n]) return;
+        if (c >= s_Q[n]) { finish(true); return; }
         const int r = find_region(s_Q, n, c);      // largest r with s_Q[r] <= c: the region this CTA cuts
         const int pieces = s_Q[r + 1] - s_Q[r], j = c - s_Q[r], units = s_P[r + 1] - s_P[r];
         u0 = s_P[r] + small_div(units * j, pieces);          // units * pieces < 2^24: both are at most a few thousand
@@ -297,7 +331,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         u0 = min(total, (int)blockIdx.x * upc);
         u1 = min(total, u0 + upc);
     }
-    if (u0 >= u1) return;
+    if (u0 >= u1) { finish(true); return; }
     DECODE_TRACE(1);
     // CTAs that hold a piece of region r, and the partial slot CTA c uses for it
     auto span_of = [&](int r, int &c0, int &c1) {
@@ -354,6 +388,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int G = p.G;
 
     int n_flush = 0;  // flushes done so far (trace slots only)
+    int len = 0;      // rows of the item being processed
     uint32_t qa[D / 16][4];
     float oacc[D / 8][4];
     float m_run[2], l_run[2];
@@ -375,8 +410,115 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         l_run[0] = l_run[1] = 0.f;
     };
 
+    // One block of 16 keys at rows blk_row0.. of a (K, V) tile in shared memory; the block's first key is row j0
+    // of the region, which has len rows.  sub_stride is the distance between the two 64-channel halves.
+    auto process_block = [&](uint32_t k_base, uint32_t v_base, uint32_t sub_stride, int blk_row0, int j0, int len) {
+        const int mi = lane >> 3, rr = lane & 7;
+
+        // ---- S = Q K^T for 16 keys ----
+        float sacc[2][4];
+#pragma unroll
+        for (int a = 0; a < 2; ++a) sacc[a][0] = sacc[a][1] = sacc[a][2] = sacc[a][3] = 0.f;
+        {
+            const int row = blk_row0 + (mi >> 1) * 8 + rr;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const int hf = kk >> 2, chunk = ((kk & 3) << 1) + (mi & 1);
+                uint32_t b[4];
+                ldmatrix_x4(b, k_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
+                mma_bf16_16816(sacc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[0], b[1]);
+                mma_bf16_16816(sacc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[2], b[3]);
+            }
+        }
+        // ---- online softmax (exp2 domain) ----
+        const bool tail = j0 + 16 > len;
+        uint32_t pa[4], pb[4];  // P = pa + pb: bf16 head and bf16 remainder of every probability
+        float corr[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            if (i >= NROW) { pa[i] = pa[i + 2] = pb[i] = pb[i + 2] = 0u; corr[i] = 1.f; continue; }
+            float x[4];
+            x[0] = sacc[0][2 * i] * p.sl2; x[1] = sacc[0][2 * i + 1] * p.sl2;
+            x[2] = sacc[1][2 * i] * p.sl2; x[3] = sacc[1][2 * i + 1] * p.sl2;
+            if (tail) {
+                const int jk = j0 + 2 * t;
+                if (jk >= len) x[0] = -INFINITY;
+                if (jk + 1 >= len) x[1] = -INFINITY;
+                if (jk + 8 >= len) x[2] = -INFINITY;
+                if (jk + 9 >= len) x[3] = -INFINITY;
+            }
+            float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float mn = fmaxf(m_run[i], mx);  // finite: row j0 of the block is valid
+            corr[i] = exp2_or_zero(m_run[i], mn);
+            m_run[i] = mn;
+            const float e0 = fast_exp2(x[0] - mn), e1 = fast_exp2(x[1] - mn);
+            const float e2 = fast_exp2(x[2] - mn), e3 = fast_exp2(x[3] - mn);
+            pa[i] = pack_bf16(e0, e1);
+            pa[i + 2] = pack_bf16(e2, e3);
+            pb[i] = pack_bf16(e0 - bf16lo(pa[i]), e1 - bf16hi(pa[i]));
+            pb[i + 2] = pack_bf16(e2 - bf16lo(pa[i + 2]), e3 - bf16hi(pa[i + 2]));
+            l_run[i] = l_run[i] * corr[i] + ((e0 + e1) + (e2 + e3));
+        }
+        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+            for (int nd = 0; nd < D / 8; ++nd) {
+                oacc[nd][0] *= corr[0]; oacc[nd][1] *= corr[0];
+                if (G_HI) { oacc[nd][2] *= corr[1]; oacc[nd][3] *= corr[1]; }
+            }
+        }
+        // ---- O += P V ----
+        uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
+        if (tail) {
+            // rows past the region's end may hold anything (slack is never written): clear them so that
+            // 0 * garbage cannot turn into NaN
+            const int jk = j0 + 2 * t;
+            vmask0 = (jk < len ? 0x0000ffffu : 0u) | (jk + 1 < len ? 0xffff0000u : 0u);
+            vmask1 = (jk + 8 < len ? 0x0000ffffu : 0u) | (jk + 9 < len ? 0xffff0000u : 0u);
+        }
+        {
+            const int row = blk_row0 + (mi & 1) * 8 + rr;
+#pragma unroll
+            for (int n2 = 0; n2 < D / 16; ++n2) {
+                const int cg = n2 * 2 + (mi >> 1);
+                const int hf = cg >> 3, chunk = cg & 7;
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, v_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
+                if (tail) { b[0] &= vmask0; b[1] &= vmask1; b[2] &= vmask0; b[3] &= vmask1; }
+                mma_bf16_16816(oacc[2 * n2], pa[0], pa[1], pa[2], pa[3], b[0], b[1]);
+                mma_bf16_16816(oacc[2 * n2 + 1], pa[0], pa[1], pa[2], pa[3], b[2], b[3]);
+                mma_bf16_16816(oacc[2 * n2], pb[0], pb[1], pb[2], pb[3], b[0], b[1]);
+                mma_bf16_16816(oacc[2 * n2 + 1], pb[0], pb[1], pb[2], pb[3], b[2], b[3]);
+            }
+        }
+    };
+
     // Writes the region's result (whole region inside this CTA) or an unnormalised partial.
     auto flush = [&](int r, int ustart, int uend) {
+        if (p.k_new != nullptr && uend == s_P[r + 1]) {
+            // Eq. 2: this CTA holds the item's last unit, so the appended token joins here.  Warp ks = 0 of every
+            // head copies the token's K and V rows into a one-row tile in the scratch area (rows 1..15 of that
+            // tile are whatever lies behind it: masked like any row past the end), stores them into the cache
+            // and runs the block routine on it.
+            if (ks == 0) {
+                const int reg = r / hs, head = HS ? r % hs : g;
+                uint8_t *area = reinterpret_cast<uint8_t *>(s_merge) + g * (4 * 128);
+                const int64_t src = ((int64_t)reg * p.kv_heads + head) * D;
+                const int64_t dst = (((int64_t)s_off[r] + len) * p.kv_heads + head) * D;
+                const int c = lane & 15;
+                if (c < D / 8) {
+                    const uint16_t *from = lane < 16 ? p.k_new : p.v_new;
+                    uint16_t *to = lane < 16 ? p.k_cache : p.v_cache;
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(from + src) + c);
+                    *reinterpret_cast<uint4 *>(area + (lane < 16 ? 0 : 2 * 128) + (c >> 3) * 128 + (c & 7) * 16) = v;
+                    reinterpret_cast<uint4 *>(to + dst)[c] = v;
+                }
+                __syncwarp();
+                process_block(smem_u32(area), smem_u32(area + 2 * 128), 128, 0, len, len + 1);
+            }
+            consumer_bar(NCW * 32);   // the scratch area becomes the merge buffer below
+        }
 #pragma unroll
         for (int i = 0; i < NROW; ++i) {
             l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
@@ -564,7 +706,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     int r = find_region(s_P, n, u0);
     int seg_start = u0;
-    int len = p.lens[r / hs];
+    len = p.lens[r / hs];
     load_q(r);
     int it = 0;
     bool ok = true;
@@ -586,92 +728,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int j0 = (u - s_P[r]) * CH + ks * 16;  // first row of this warp's block inside the region
         if (j0 < len) {
             const uint32_t k_base = smem_u32(s_stage + s * C::STAGE_BYTES) + g * C::HALVES * C::SUBTILE;
-            const uint32_t v_base = k_base + C::KV_BYTES;
-            const int mi = lane >> 3, rr = lane & 7;
-
-            // ---- S = Q K^T for 16 keys ----
-            float sacc[2][4];
-#pragma unroll
-            for (int a = 0; a < 2; ++a) sacc[a][0] = sacc[a][1] = sacc[a][2] = sacc[a][3] = 0.f;
-            {
-                const int row = ks * 16 + (mi >> 1) * 8 + rr;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const int hf = kk >> 2, chunk = ((kk & 3) << 1) + (mi & 1);
-                    uint32_t b[4];
-                    ldmatrix_x4(b, k_base + hf * C::SUBTILE + row * 128 + ((chunk ^ (row & 7)) << 4));
-                    mma_bf16_16816(sacc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[0], b[1]);
-                    mma_bf16_16816(sacc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[2], b[3]);
-                }
-            }
-            // ---- online softmax (exp2 domain) ----
-            const bool tail = j0 + 16 > len;
-            uint32_t pa[4], pb[4];  // P = pa + pb: bf16 head and bf16 remainder of every probability
-            float corr[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                if (i >= NROW) { pa[i] = pa[i + 2] = pb[i] = pb[i + 2] = 0u; corr[i] = 1.f; continue; }
-                float x[4];
-                x[0] = sacc[0][2 * i] * p.sl2; x[1] = sacc[0][2 * i + 1] * p.sl2;
-                x[2] = sacc[1][2 * i] * p.sl2; x[3] = sacc[1][2 * i + 1] * p.sl2;
-                if (tail) {
-                    const int jk = j0 + 2 * t;
-                    if (jk >= len) x[0] = -INFINITY;
-                    if (jk + 1 >= len) x[1] = -INFINITY;
-                    if (jk + 8 >= len) x[2] = -INFINITY;
-                    if (jk + 9 >= len) x[3] = -INFINITY;
-                }
-                float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float mn = fmaxf(m_run[i], mx);  // finite: row j0 of the block is valid
-                corr[i] = exp2_or_zero(m_run[i], mn);
-                m_run[i] = mn;
-                const float e0 = fast_exp2(x[0] - mn), e1 = fast_exp2(x[1] - mn);
-                const float e2 = fast_exp2(x[2] - mn), e3 = fast_exp2(x[3] - mn);
-                pa[i] = pack_bf16(e0, e1);
-                pa[i + 2] = pack_bf16(e2, e3);
-                pb[i] = pack_bf16(e0 - bf16lo(pa[i]), e1 - bf16hi(pa[i]));
-                pb[i + 2] = pack_bf16(e2 - bf16lo(pa[i + 2]), e3 - bf16hi(pa[i + 2]));
-                l_run[i] = l_run[i] * corr[i] + ((e0 + e1) + (e2 + e3));
-            }
-            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-                for (int nd = 0; nd < D / 8; ++nd) {
-                    oacc[nd][0] *= corr[0]; oacc[nd][1] *= corr[0];
-                    if (G_HI) { oacc[nd][2] *= corr[1]; oacc[nd][3] *= corr[1]; }
-                }
-            }
-            // ---- O += P V ----
-            uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
-            if (tail) {
-                // rows past the region's end may hold anything (slack is never written): clear them so that
-                // 0 * garbage cannot turn into NaN
-                const int jk = j0 + 2 * t;
-                vmask0 = (jk < len ? 0x0000ffffu : 0u) | (jk + 1 < len ? 0xffff0000u : 0u);
-                vmask1 = (jk + 8 < len ? 0x0000ffffu : 0u) | (jk + 9 < len ? 0xffff0000u : 0u);
-            }
-            {
-                const int row = ks * 16 + (mi & 1) * 8 + rr;
-#pragma unroll
-                for (int n2 = 0; n2 < D / 16; ++n2) {
-                    const int cg = n2 * 2 + (mi >> 1);
-                    const int hf = cg >> 3, chunk = cg & 7;
-                    uint32_t b[4];
-                    ldmatrix_x4_trans(b, v_base + hf * C::SUBTILE + row * 128 + ((chunk ^ (row & 7)) << 4));
-                    if (tail) { b[0] &= vmask0; b[1] &= vmask1; b[2] &= vmask0; b[3] &= vmask1; }
-                    mma_bf16_16816(oacc[2 * n2], pa[0], pa[1], pa[2], pa[3], b[0], b[1]);
-                    mma_bf16_16816(oacc[2 * n2 + 1], pa[0], pa[1], pa[2], pa[3], b[2], b[3]);
-                    mma_bf16_16816(oacc[2 * n2], pb[0], pb[1], pb[2], pb[3], b[0], b[1]);
-                    mma_bf16_16816(oacc[2 * n2 + 1], pb[0], pb[1], pb[2], pb[3], b[2], b[3]);
-                }
-            }
+            process_block(k_base, k_base + C::KV_BYTES, C::SUBTILE, ks * 16, j0, len);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_bar[kStages + s]));
     }
     DECODE_TRACE(3 + 3 * n_flush);
     if (ok) flush(r, seg_start, u1);
+    finish(false);
     DECODE_TRACE(5 + 3 * n_flush);
     DECODE_TRACE(15);
     (void)n_flush;
@@ -764,8 +828,8 @@ int launch_decode_d(const aircache_shape_t *s, const aircache_ragged_t *c, Decod
 
 }  // namespace
 
-int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out, void *ws,
-                  cudaStream_t st) {
+int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, const void *k_new,
+                  const void *v_new, float *out, void *ws, cudaStream_t st) {
     const WsLayout w = ws_layout(s);
     DecodeParams p;
     p.q = (const uint16_t *)q;
@@ -775,6 +839,13 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.tickets = ws_ptr<int32_t>(ws, w.tickets);
     p.partials = ws_ptr<float>(ws, w.partials);
     p.status = ws_ptr<uint32_t>(ws, w.status);
+    p.k_new = (const uint16_t *)k_new;
+    p.v_new = (const uint16_t *)v_new;
+    p.k_cache = (uint16_t *)c->k;
+    p.v_cache = (uint16_t *)c->v;
+    p.lens_rw = c->lens;
+    p.done_ticket = ws_ptr<int32_t>(ws, w.status) + 4;   // fifth word of the status block
+    p.kv_heads = s->n_kv_heads;
     p.n_regions = s->n_layers * s->batch;
     p.Hq = s->n_q_heads;
     p.G = s->n_q_heads / s->n_kv_heads;
@@ -825,6 +896,11 @@ int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, 
     p.offsets = c->offsets;
     p.lens = c->lens;
     p.status = reinterpret_cast<uint32_t *>(base);
+    p.k_new = p.v_new = nullptr;
+    p.k_cache = p.v_cache = nullptr;
+    p.lens_rw = nullptr;
+    p.done_ticket = nullptr;
+    p.kv_heads = s->n_kv_heads;
     p.tickets = reinterpret_cast<int32_t *>(base + 256);
     p.partials = reinterpret_cast<float *>(base + kStatusBytes);
     p.n_regions = s->n_layers * s->batch;

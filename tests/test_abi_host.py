@@ -21,7 +21,7 @@ def declared_functions():
 
 def test_library_exports_every_declared_symbol():
     names = declared_functions()
-    assert len(names) >= 14
+    assert len(names) >= 15
     handle = C.CDLL(ac.LIB)
     for n in names:
         assert hasattr(handle, n), f"{n} declared in aircache.h but not exported"
@@ -119,6 +119,9 @@ def test_entry_points_reject_bad_arguments_on_the_host():
     assert ac.aircache_decode_attn(sh, rag, P, P + 4, ws, s, check=False) == ac.ERR_ALIGNMENT
     assert ac.aircache_decode_attn(sh, ac.Ragged(None, P, P, P, 10), P, P, ws, s, check=False) == ac.ERR_INVALID_ARG
     assert ac.aircache_decode_attn(sh, ac.Ragged(P, P, P, P, 0), P, P, ws, s, check=False) == ac.ERR_CAPACITY
+    # fused step: slack is 0, so the append overflows; NULL token
+    assert ac.aircache_decode_step(sh, rag, P, P, P, 0, P, ws, s, check=False) == ac.ERR_CAPACITY
+    assert ac.aircache_decode_step(sh, rag, P, None, P, 0, P, ws, s, check=False) == ac.ERR_INVALID_ARG
     # append: slack is 0, so any append overflows
     assert ac.aircache_append(sh, rag, P, P, 0, s, check=False) == ac.ERR_CAPACITY
     # status helpers

@@ -31,6 +31,8 @@ CASES = {
     "kv1": small("kv1", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=130, Nt=9, W=9),
     # long regions cut across many CTAs with an odd head count (padded partial slots, multi-round merge)
     "kv1long": small("kv1long", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=9000, Nt=9, W=4, ratio=0.9),
+    # more (region, KV head) pairs than SMs: the by-region decode schedule with several regions per CTA
+    "many": small("many", L=10, Hq=28, Hkv=4, d=128, B=4, Nv=300, Nt=20, W=8),
 }
 
 
@@ -363,6 +365,43 @@ def test_append_then_decode(oracle):
     want = oracle.decode(ref["dims"], k_o, v_o, cp["offsets"], lens, u16(q), wl.scale)
     gp.decode(q.to(DEV))
     assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+
+
+@pytest.mark.parametrize("case", ["s7b", "c1", "s72b", "kv1long", "many"])
+def test_fused_decode_step_appends_and_attends(oracle, case):
+    """aircache_decode_step: the new token's K/V land in the slack rows, take part in the same call's attention,
+    and lens grows - checked against the oracle on the cache extended by hand, three steps in a row."""
+    import paper_2503_23956_b200 as ac
+    wl = CASES[case]
+    slack = 3
+    ref = oracle_path(oracle, wl, slack=slack)
+    cp = ref["compact"]
+    gp = make_gpu(wl, ref, slack=slack)
+    run_chain(gp, ref)
+    rng = np.random.default_rng(17)
+    k_o, v_o, lens = cp["k"].copy(), cp["v"].copy(), cp["lens"].copy()
+    LB = wl.n_layers * wl.batch
+    for i in range(slack):
+        kn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        vn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        for r in range(LB):
+            k_o[cp["offsets"][r] + lens[r]] = u16(kn)[r]
+            v_o[cp["offsets"][r] + lens[r]] = u16(vn)[r]
+        lens += 1
+        q = decode_queries(wl, i, "cpu")
+        want = oracle.decode(ref["dims"], k_o, v_o, cp["offsets"], lens, u16(q), wl.scale)
+        gp.out.fill_(float("nan"))
+        ac.aircache_decode_step(gp.sh, gp.cache, q.to(DEV), kn.to(DEV), vn.to(DEV), i, gp.out, gp.ws)
+        assert gp.status() == 0
+        assert np.array_equal(gp.lens.cpu().numpy(), lens)
+        assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+    # the appended rows are in the cache, bit for bit
+    kc, vc = u16(gp.k_c), u16(gp.v_c)
+    for r in range(LB):
+        a, n = int(cp["offsets"][r]), int(lens[r])
+        assert np.array_equal(kc[a:a + n], k_o[a:a + n]) and np.array_equal(vc[a:a + n], v_o[a:a + n])
+    assert ac.aircache_decode_step(gp.sh, gp.cache, q.to(DEV), kn.to(DEV), vn.to(DEV), slack, gp.out, gp.ws,
+                                   check=False) == ac.ERR_CAPACITY
 
 
 def test_pipeline_host_matches_staged_calls(oracle):
