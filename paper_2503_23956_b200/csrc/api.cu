@@ -70,9 +70,6 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.group_ticket = take(groups * 4);
     w.mom_strength = take(LB * 8);
     w.mom_skew = take(LB * 8);
-    w.alloc_w = take(LB * 8);
-    w.alloc_share = take(LB * 8);
-    w.alloc_active = take(LB * 4);
     w.kept = take(LB * s->n_visual * 4);
     w.partials = take((int64_t)2 * kMaxDecodeCtas * partial_slot_floats(s->n_q_heads, s->head_dim) * 4);
     w.total = off;

@@ -92,9 +92,6 @@ struct WsLayout {
     int64_t group_ticket; // u32  [L*B*Hkv]            chunks of the group done so far
     int64_t mom_strength; // f64  [L*B]
     int64_t mom_skew;     // f64  [L*B]
-    int64_t alloc_w;      // f64  [L*B]
-    int64_t alloc_share;  // f64  [L*B]
-    int64_t alloc_active; // i32  [L*B]
     int64_t kept;         // i32  [L*B*Nv]             kept-token lists when the caller passes none
     int64_t partials;     // f32  [2*kMaxDecodeCtas][Hq*(d+2)]
     int64_t total;

@@ -7,7 +7,7 @@ import torch
 
 import paper_2503_23956_b200 as ac
 from paper_2503_23956_b200.session import Session
-from workloads import decode_queries, full_cache, window_queries
+from workloads import full_cache, window_queries
 from workloads.synth import to_u16
 
 
