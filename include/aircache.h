@@ -258,6 +258,16 @@ int aircache_reset_status(void *workspace, int64_t workspace_bytes, void *cuda_s
 int aircache_check_status(void *workspace, int64_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Diagnostics: enqueues a one-CTA kernel whose threads wait, with the same
+ * bounded wait the decode kernel uses, on a barrier that nothing completes.
+ * The wait gives up after its poll limit (a fraction of a second), the kernel
+ * returns normally and the workspace's status word is set, so a following
+ * aircache_check_status() reports AIRCACHE_ERR_TIMEOUT; aircache_reset_status()
+ * clears it.  Shows that a stuck wait ends in an error code, not in a hang.
+ */
+int aircache_selftest_wait_timeout(void *workspace, int64_t workspace_bytes, void *cuda_stream);
+
+/*
  * The whole path with HOST inputs and outputs: uploads the full cache and the
  * queries, runs score -> budget -> compact -> n_steps x decode_attn on the
  * stream, downloads the results and synchronises.  Every device buffer is still

@@ -74,6 +74,7 @@ _SIGNATURES = {
                                   C.c_void_p]),
     "aircache_reset_status": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_check_status": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
+    "aircache_selftest_wait_timeout": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_pipeline_host": (C.c_int, [C.POINTER(Shape), C.POINTER(Full), C.c_int64, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float,
                                          C.c_double, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(Ragged),
@@ -233,6 +234,13 @@ def aircache_check_status(workspace, stream=None, check=True) -> int:
     rc = lib().aircache_check_status(_ptr(workspace), _nbytes(workspace), _stream(stream))
     if check:
         _check("aircache_check_status", rc)
+    return rc
+
+
+def aircache_selftest_wait_timeout(workspace, stream=None, check=True) -> int:
+    rc = lib().aircache_selftest_wait_timeout(_ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check("aircache_selftest_wait_timeout", rc)
     return rc
 
 

@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace aircache {
 
@@ -92,6 +93,31 @@ static int check_ragged(const aircache_shape_t *s, const aircache_ragged_t *c, b
         if (c->total_rows < 1 || c->total_rows >= ((int64_t)1 << 31)) return AIRCACHE_ERR_CAPACITY;
     }
     (void)s;
+    return AIRCACHE_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// aircache_selftest_wait_timeout: the bounded wait on a barrier that nobody completes
+// ---------------------------------------------------------------------------------------------
+namespace {
+__global__ void wait_timeout_kernel(uint32_t *status) {
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&s_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_abort = 0;
+    }
+    __syncthreads();
+    // no thread ever arrives: every waiter gives up after kSpinLimit polls (or as soon as one of them has),
+    // the first one records the status word
+    mbar_wait(smem_u32(&s_bar), 0, &s_abort, status, 9);
+}
+}  // namespace
+
+int launch_selftest_timeout(void *ws, cudaStream_t st) {
+    wait_timeout_kernel<<<1, 64, 0, st>>>(reinterpret_cast<uint32_t *>(ws));
+    AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }
 
@@ -250,6 +276,13 @@ int aircache_check_status(void *workspace, int64_t workspace_bytes, void *cuda_s
                                       (cudaStream_t)cuda_stream));
     AIRCACHE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
     return word ? AIRCACHE_ERR_TIMEOUT : AIRCACHE_OK;
+}
+
+int aircache_selftest_wait_timeout(void *workspace, int64_t workspace_bytes, void *cuda_stream) {
+    if (!workspace) return AIRCACHE_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace & 255) return AIRCACHE_ERR_ALIGNMENT;
+    if (workspace_bytes < kStatusBytes) return AIRCACHE_ERR_WORKSPACE_TOO_SMALL;
+    return launch_selftest_timeout(workspace, (cudaStream_t)cuda_stream);
 }
 
 int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t *h_full, int64_t full_elems,

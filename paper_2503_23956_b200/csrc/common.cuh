@@ -116,6 +116,7 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
                   const void *v_new, float *out, void *ws, cudaStream_t st);
 int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, float *out,
                          cudaStream_t st);
+int launch_selftest_timeout(void *ws, cudaStream_t st);
 int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,
                   int32_t appended, cudaStream_t st);
 

@@ -9,7 +9,7 @@
 
 namespace aircache {
 
-constexpr uint32_t kSpinLimit = 1u << 22;   // polls before a bounded mbarrier wait gives up
+constexpr uint32_t kSpinLimit = 1u << 18;   // polls before a bounded mbarrier wait gives up (about a second)
 
 // ---------------------------------------------------------------------------------------------
 // host: cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)

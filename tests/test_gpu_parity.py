@@ -404,6 +404,28 @@ def test_fused_decode_step_appends_and_attends(oracle, case):
                                    check=False) == ac.ERR_CAPACITY
 
 
+def test_bounded_wait_ends_in_an_error_code_not_a_hang():
+    """A wait that nothing satisfies gives up after its poll limit: the kernel returns, the status word is set,
+    aircache_check_status reports the timeout, a reset clears it and the workspace is usable again."""
+    import time
+    import paper_2503_23956_b200 as ac
+    wl = CASES["c1"]
+    gp = GpuPath(wl, device=DEV)
+    assert gp.status() == 0
+    t0 = time.time()
+    ac.aircache_selftest_wait_timeout(gp.ws)
+    assert gp.status() == ac.ERR_TIMEOUT
+    assert time.time() - t0 < 20.0
+    ac.aircache_reset_status(gp.ws)
+    assert gp.status() == 0
+    # the context is intact: a normal decode still works afterwards
+    k, v, qw = gen_inputs(wl, DEV)
+    gp.set_full(logical(k), logical(v))
+    gp.score(qw); gp.budget(); gp.compact()
+    gp.decode(decode_queries(wl, 0, DEV))
+    assert gp.status() == 0 and torch.isfinite(gp.out).all()
+
+
 def test_pipeline_host_matches_staged_calls(oracle):
     import paper_2503_23956_b200 as ac
     wl = CASES["c1"]
