@@ -404,6 +404,61 @@ def test_fused_decode_step_appends_and_attends(oracle, case):
                                    check=False) == ac.ERR_CAPACITY
 
 
+def _random_workload(seed):
+    rng = np.random.default_rng(1000 + seed)
+    hkv = int(rng.choice([1, 2, 4, 8]))
+    g = int(rng.choice([1, 2, 3, 4, 7, 8, 12, 16]))
+    d = int(rng.choice([64, 128]))
+    L = int(rng.integers(1, 6))
+    B = int(rng.integers(1, 4))
+    nv = int(rng.choice([3, 4, 7, 15, 16, 17, 31, 33, 64, 100, 129, 255, 300, 513, 700]))
+    nt = int(rng.choice([1, 2, 3, 5, 16, 17, 40, 70]))
+    W = int(rng.integers(1, min(nt, 64) + 1))
+    ratio = float(rng.choice([0.0, 0.05, 0.1, 0.33, 0.5, 0.9, 1.0]))
+    alpha = float(rng.choice([0.0, 0.5, 0.9, 0.99, 1.0]))
+    slack = int(rng.choice([0, 1, 2, 5]))
+    return small(f"rnd{seed}", L=L, Hq=hkv * g, Hkv=hkv, d=d, B=B, Nv=nv, Nt=nt, W=W, ratio=ratio, alpha=alpha), slack
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shapes_whole_chain(oracle, seed):
+    """Seeded random shapes (head layouts, head_dim, tiny and ragged token counts, window sizes, retention 0..1,
+    thresholds 0..1, slack): the whole chain, one decode and - when there is slack - one fused decode step."""
+    import paper_2503_23956_b200 as ac
+    wl, slack = _random_workload(seed)
+    ref = oracle_path(oracle, wl, slack=slack)
+    cp = ref["compact"]
+    gp = make_gpu(wl, ref, slack=slack)
+    run_chain(gp, ref)
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"]), wl
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL, wl
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"]), wl
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"]), wl
+    compare_cache(gp, cp)
+    q = decode_queries(wl, 0, "cpu")
+    want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q), wl.scale)
+    gp.out.fill_(float("nan"))
+    gp.decode(q.to(DEV))
+    assert gp.status() == 0
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL, wl
+    if slack > 0:
+        rng = np.random.default_rng(seed)
+        LB = wl.n_layers * wl.batch
+        kn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        vn = torch.from_numpy(rng.standard_normal((LB, wl.n_kv_heads, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+        k_o, v_o, lens = cp["k"].copy(), cp["v"].copy(), cp["lens"].copy()
+        for r in range(LB):
+            k_o[cp["offsets"][r] + lens[r]] = u16(kn)[r]
+            v_o[cp["offsets"][r] + lens[r]] = u16(vn)[r]
+        lens += 1
+        q1 = decode_queries(wl, 1, "cpu")
+        want = oracle.decode(ref["dims"], k_o, v_o, cp["offsets"], lens, u16(q1), wl.scale)
+        ac.aircache_decode_step(gp.sh, gp.cache, q1.to(DEV), kn.to(DEV), vn.to(DEV), 0, gp.out, gp.ws)
+        assert gp.status() == 0
+        assert np.array_equal(gp.lens.cpu().numpy(), lens)
+        assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL, wl
+
+
 def test_bounded_wait_ends_in_an_error_code_not_a_hang():
     """A wait that nothing satisfies gives up after its poll limit: the kernel returns, the status word is set,
     aircache_check_status reports the timeout, a reset clears it and the workspace is usable again."""
