@@ -100,6 +100,8 @@ struct DecodeCfg {
     static constexpr int NROW = G_HI ? 2 : 1;        // accumulator row groups in use (heads 0-7, heads 8-15)
     static constexpr int KSPLIT = HS ? 8 : ((8 / HKV) > 4 ? 4 : (8 / HKV));
     static constexpr int CH = 16 * KSPLIT;           // rows per unit
+    static constexpr int CH_LOG2 = KSPLIT == 8 ? 7 : (KSPLIT == 4 ? 6 : (KSPLIT == 2 ? 5 : 4));
+    static_assert((1 << CH_LOG2) == CH, "unit rows are a power of two");
     static constexpr int NCW = HKV * KSPLIT;         // consumer warps
     static constexpr int THREADS = (NCW + 1) * 32;
     static constexpr int HALVES = D / 64;
@@ -144,6 +146,111 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
     return lo;
 }
 
+// The region-aligned cut for few regions, planned by one warp in registers (all warps of a CTA call this and
+// get the same answer).  With no more items than CTAs a CTA needs five numbers of the cut: its item, the
+// item's units and rows, its piece and the piece count.  Each lane takes rpl consecutive regions; sums and the
+// prefix of the piece counts go through warp primitives, so no warp waits for another, no table is built, and
+// the producer can issue its first loads one global round trip after the kernel may read memory.
+// Returns 0 when the tables have to decide (empty regions, too many regions, no fitting cut), 2 when this CTA
+// has no piece, 1 with plan = {item, rows of the item, first unit, end unit} and the item's table entries
+// stored (units counted from the item's first one).
+__device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64_t *offsets, int n, int hs, int n_ctas,
+                                                int ch_log2, int c, int *s_P, int *s_off, int *s_Q, int4 *plan) {
+    constexpr int RPL = kMaxDecodeCtas / 32;
+    const int lane = threadIdx.x & 31;
+    const int nr = n / hs;
+    if (n > n_ctas || nr <= 0 || nr > 32 * RPL) return 0;
+    const int rpl = (nr + 31) >> 5;
+    int un[RPL], ln[RPL], of[RPL];
+    bool nonempty = true;
+    int tot = 0;
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        un[j] = ln[j] = of[j] = 0;
+        const int reg = lane * rpl + j;
+        if (j < rpl && reg < nr) {
+            ln[j] = max(lens[reg], 0);
+            of[j] = (int)offsets[reg];
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        const int reg = lane * rpl + j;
+        if (j < rpl && reg < nr) {
+            un[j] = (ln[j] + (1 << ch_log2) - 1) >> ch_log2;
+            nonempty = nonempty && un[j] > 0;
+            tot += un[j];
+        }
+    }
+    tot = __reduce_add_sync(0xffffffffu, tot);   // units of one head's items
+    if (!__all_sync(0xffffffffu, nonempty) || tot >= (1 << 22) / hs) return 0;
+    const int upc = max(1, small_div(tot * hs + n_ctas - 1, n_ctas));
+    // pieces of at most upc_a units: the smallest of upc, upc + 1, upc + 2 that needs no more CTAs than there are
+    int sum0 = 0, sum1 = 0, sum2 = 0;
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        if (j < rpl) {
+            sum0 += small_div(un[j] + upc - 1, upc);
+            sum1 += small_div(un[j] + upc, upc + 1);
+            sum2 += small_div(un[j] + upc + 1, upc + 2);
+        }
+    }
+    sum0 = __reduce_add_sync(0xffffffffu, sum0);
+    sum1 = __reduce_add_sync(0xffffffffu, sum1);
+    sum2 = __reduce_add_sync(0xffffffffu, sum2);
+    const int lim = n_ctas / hs;   // the sums count pieces per head
+    if (sum0 > lim && sum1 > lim && sum2 > lim) return 0;
+    const int upc_a = sum0 <= lim ? upc : (sum1 <= lim ? upc + 1 : upc + 2);
+    int pc[RPL];
+    int mine = 0;
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        pc[j] = j < rpl ? small_div(un[j] + upc_a - 1, upc_a) : 0;
+        mine += pc[j];
+    }
+    int incl = mine;
+#pragma unroll
+    for (int sh = 1; sh < 32; sh <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+        if (lane >= sh) incl += o;
+    }
+    // the region whose CTAs [first * hs, (first + pieces) * hs) include this one
+    int run = incl - mine;
+    int v_reg = -1, v_first = 0, v_pc = 0, v_un = 0, v_ln = 0, v_of = 0;
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        if (j < rpl) {
+            if (c >= run * hs && c < (run + pc[j]) * hs) {
+                v_reg = lane * rpl + j; v_first = run; v_pc = pc[j]; v_un = un[j]; v_ln = ln[j]; v_of = of[j];
+            }
+            run += pc[j];
+        }
+    }
+    const unsigned ball = __ballot_sync(0xffffffffu, v_reg >= 0);
+    if (ball == 0) return 2;   // more CTAs than pieces
+    const int src = __ffs(ball) - 1;
+    v_reg = __shfl_sync(0xffffffffu, v_reg, src);
+    v_first = __shfl_sync(0xffffffffu, v_first, src);
+    v_pc = __shfl_sync(0xffffffffu, v_pc, src);
+    v_un = __shfl_sync(0xffffffffu, v_un, src);
+    v_ln = __shfl_sync(0xffffffffu, v_ln, src);
+    v_of = __shfl_sync(0xffffffffu, v_of, src);
+    const int rel = c - v_first * hs;
+    const int h = small_div(rel, v_pc), j = rel - h * v_pc;
+    const int item = v_reg * hs + h;
+    // no overflow: the units of all regions together are below 2^22, the pieces at most 256
+    *plan = make_int4(item, v_ln, small_div(v_un * j, v_pc), small_div(v_un * (j + 1), v_pc));
+    if (lane == 0) {
+        s_P[item] = 0;
+        s_P[item + 1] = v_un;
+        s_off[item] = v_of;
+        s_Q[item] = v_first * hs + h * v_pc;
+        s_Q[item + 1] = v_first * hs + (h + 1) * v_pc;
+    }
+    __syncwarp();
+    return 1;
+}
+
 template <int D, int HKV, bool G_HI, bool HS>
 __global__ void __launch_bounds__(DecodeCfg<D, HKV, G_HI, HS>::THREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, DecodeParams p) {
@@ -185,128 +292,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s_abort = 0;
     }
+    // The barriers are initialised before any warp goes its own way (nothing above read global memory).
+    __syncthreads();
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // ---- unit prefix and first row of all regions (every CTA computes the same tables) ----
-    {
-        const int per = (n + C::THREADS - 1) / C::THREADS;
-        const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
-        int local = 0;
-        for (int i = i0; i < i1; ++i) {
-            local += (max(p.lens[i / hs], 0) + CH - 1) / CH;
-            s_off[i] = (int)p.offsets[i / hs];
-        }
-        s_part[tid] = local;
-        __syncthreads();
-        DECODE_TRACE(12);
-        if (wid == 0) {
-            // warp 0 turns s_part into an exclusive prefix
-            constexpr int PER_LANE = (C::THREADS + 31) / 32;
-            int sum = 0;
-            for (int j = 0; j < PER_LANE; ++j) {
-                const int idx = lane * PER_LANE + j;
-                if (idx < C::THREADS) sum += s_part[idx];
-            }
-            int incl = sum;
-#pragma unroll
-            for (int sh = 1; sh < 32; sh <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, sh);
-                if (lane >= sh) incl += o;
-            }
-            int run = incl - sum;
-            for (int j = 0; j < PER_LANE; ++j) {
-                const int idx = lane * PER_LANE + j;
-                if (idx < C::THREADS) { const int v = s_part[idx]; s_part[idx] = run; run += v; }
-            }
-        }
-        __syncthreads();
-        int run = s_part[tid];
-        for (int i = i0; i < i1; ++i) {
-            s_P[i] = run;
-            run += (max(p.lens[i / hs], 0) + CH - 1) / CH;
-        }
-        if (i1 == n && i0 < n) s_P[n] = run;
-        if (n == 0 && tid == 0) s_P[0] = 0;
-        __syncthreads();
-    }
-    DECODE_TRACE(13);
-    const int total = s_P[n];
-    const int upc = max(1, small_div(total + n_ctas - 1, n_ctas));
-
-    // ---- schedule.  Balanced mode: CTA c takes units [c * upc, (c+1) * upc) of the global list.
-    // Region-aligned mode (few regions, each cut into pieces of at most upc units, if that needs no more
-    // CTAs than there are): every CTA works on one region only, so it reloads no query and flushes once.
-    if (wid == 0) {
-        // Aligned pieces of at most upc_a units: upc_a is the smallest of upc, upc + 1, upc + 2 for which the
-        // pieces need no more CTAs than the grid has (two more units on the longest CTA cost less than a
-        // second flush and merge).  All items of a region have the same unit count, so the sums run over
-        // regions; the three candidates are evaluated together.  Rolled loops: this runs once.
-        const bool few = n <= n_ctas && total > 0;
-        const int nr = n / hs;
-        int sum0 = 0, sum1 = 0, sum2 = 0;
-#pragma unroll 1
-        for (int r = lane; few && r < nr; r += 32) {
-            const int u = s_P[r * hs + 1] - s_P[r * hs];
-            sum0 += small_div(u + upc - 1, upc);
-            sum1 += small_div(u + upc, upc + 1);
-            sum2 += small_div(u + upc + 1, upc + 2);
-        }
-#pragma unroll
-        for (int sh = 16; sh > 0; sh >>= 1) {
-            sum0 += __shfl_xor_sync(0xffffffffu, sum0, sh);
-            sum1 += __shfl_xor_sync(0xffffffffu, sum1, sh);
-            sum2 += __shfl_xor_sync(0xffffffffu, sum2, sh);
-        }
-        const int lim = n_ctas / hs;   // the sums count pieces per head
-        const bool found = few && (sum0 <= lim || sum1 <= lim || sum2 <= lim);
-        const int upc_a = sum0 <= lim ? upc : (sum1 <= lim ? upc + 1 : upc + 2);
-        int carry = 0;
-#pragma unroll 1
-        for (int base = 0; found && base <= nr; base += 32) {
-            const int r = base + lane;
-            const int v = r < nr ? small_div(s_P[r * hs + 1] - s_P[r * hs] + upc_a - 1, upc_a) : 0;
-            int incl = v;
-#pragma unroll
-            for (int sh = 1; sh < 32; sh <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, sh);
-                if (lane >= sh) incl += o;
-            }
-            if (r < nr) {
-#pragma unroll 1
-                for (int h = 0; h < hs; ++h) s_Q[r * hs + h] = (carry + incl - v) * hs + h * v;
-            } else if (r == nr) {
-                s_Q[n] = (carry + incl - v) * hs;
-            }
-            carry += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (lane == 0) s_aligned = found ? 1 : 0;
-    }
-    __syncthreads();
-    DECODE_TRACE(14);
-    const bool aligned = s_aligned != 0;
-
-    // an item without rows yields zeros - or, when a token is appended, that token's value (softmax over one key)
-    for (int r = blockIdx.x; r < n; r += n_ctas) {
-        if (s_P[r + 1] != s_P[r]) continue;
-        const int reg = r / hs;
-        for (int i = tid; i < p.Hq * D; i += C::THREADS) {
-            float v = 0.f;
-            if (p.k_new) {
-                const int kvh = HS ? r % hs : (i / D) / p.G;
-                v = bf16_to_f32(p.v_new[((int64_t)reg * p.kv_heads + kvh) * D + i % D]);
-            }
-            p.out[(int64_t)r * p.Hq * D + i] = v;
-        }
-        if (p.k_new) {
-            const int heads = HS ? 1 : p.kv_heads, h0 = HS ? r % hs : 0;
-            for (int i = tid; i < heads * D; i += C::THREADS) {
-                const int64_t src = ((int64_t)reg * p.kv_heads + h0) * D + i;
-                const int64_t dst = ((int64_t)s_off[r] * p.kv_heads + h0) * D + i;
-                p.k_cache[dst] = p.k_new[src];
-                p.v_cache[dst] = p.v_new[src];
-            }
-        }
-    }
+    int total = 0, upc = 1;
+    bool aligned = false;
+    int u0 = 0, u1 = 0;
+    int r_own = -1, len_own = 0;   // the one item of this CTA and its rows, when the register plan found them
     // Eq. 2 bookkeeping: the CTA that finishes last adds the appended token to every region's length
     auto finish = [&](bool all_threads) {
         if (p.k_new == nullptr) return;
@@ -319,17 +312,152 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         if (s_last)
             for (int i = tid; i < n / hs; i += (all_threads ? C::THREADS : NCW * 32)) p.lens_rw[i] += 1;
     };
-    int u0, u1;
-    if (aligned) {
-        const int c = (int)blockIdx.x;
-        if (c >= s_Q[n]) { finish(true); return; }
-        const int r = find_region(s_Q, n, c);      // largest r with s_Q[r] <= c: the region this CTA cuts
-        const int pieces = s_Q[r + 1] - s_Q[r], j = c - s_Q[r], units = s_P[r + 1] - s_P[r];
-        u0 = s_P[r] + small_div(units * j, pieces);          // units * pieces < 2^24: both are at most a few thousand
-        u1 = s_P[r] + small_div(units * (j + 1), pieces);
-    } else {
-        u0 = min(total, (int)blockIdx.x * upc);
-        u1 = min(total, u0 + upc);
+
+    // ---- few regions: every warp plans for itself, in registers; otherwise the tables below decide ----
+    bool planned = false;
+    if constexpr (HS) {   // head-split launches are the ones with few items; the by-region kernels keep their registers
+        int4 plan;
+        const int rc = plan_few_regions(p.lens, p.offsets, n, hs, n_ctas, C::CH_LOG2, (int)blockIdx.x, s_P, s_off, s_Q,
+                                        &plan);
+        if (rc == 2) { finish(true); return; }
+        if (rc == 1) {
+            planned = aligned = true;
+            r_own = plan.x; len_own = plan.y; u0 = plan.z; u1 = plan.w;
+        }
+    }
+    DECODE_TRACE(12);
+    if (!planned) {
+        // ---- unit prefix and first row of all regions (every CTA computes the same tables) ----
+        {
+            const int per = (n + C::THREADS - 1) / C::THREADS;
+            const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
+            int local = 0;
+            for (int i = i0; i < i1; ++i) {
+                local += (max(p.lens[i / hs], 0) + CH - 1) / CH;
+                s_off[i] = (int)p.offsets[i / hs];
+            }
+            s_part[tid] = local;
+            __syncthreads();
+            DECODE_TRACE(12);
+            if (wid == 0) {
+                // warp 0 turns s_part into an exclusive prefix
+                constexpr int PER_LANE = (C::THREADS + 31) / 32;
+                int sum = 0;
+                for (int j = 0; j < PER_LANE; ++j) {
+                    const int idx = lane * PER_LANE + j;
+                    if (idx < C::THREADS) sum += s_part[idx];
+                }
+                int incl = sum;
+    #pragma unroll
+                for (int sh = 1; sh < 32; sh <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+                    if (lane >= sh) incl += o;
+                }
+                int run = incl - sum;
+                for (int j = 0; j < PER_LANE; ++j) {
+                    const int idx = lane * PER_LANE + j;
+                    if (idx < C::THREADS) { const int v = s_part[idx]; s_part[idx] = run; run += v; }
+                }
+            }
+            __syncthreads();
+            int run = s_part[tid];
+            for (int i = i0; i < i1; ++i) {
+                s_P[i] = run;
+                run += (max(p.lens[i / hs], 0) + CH - 1) / CH;
+            }
+            if (i1 == n && i0 < n) s_P[n] = run;
+            if (n == 0 && tid == 0) s_P[0] = 0;
+            __syncthreads();
+        }
+        DECODE_TRACE(13);
+        total = s_P[n];
+        upc = max(1, small_div(total + n_ctas - 1, n_ctas));
+
+        // ---- schedule.  Balanced mode: CTA c takes units [c * upc, (c+1) * upc) of the global list.
+        // Region-aligned mode (few regions, each cut into pieces of at most upc units, if that needs no more
+        // CTAs than there are): every CTA works on one region only, so it reloads no query and flushes once.
+        if (wid == 0) {
+            // Aligned pieces of at most upc_a units: upc_a is the smallest of upc, upc + 1, upc + 2 for which the
+            // pieces need no more CTAs than the grid has (two more units on the longest CTA cost less than a
+            // second flush and merge).  All items of a region have the same unit count, so the sums run over
+            // regions; the three candidates are evaluated together.  Rolled loops: this runs once.
+            const bool few = n <= n_ctas && total > 0;
+            const int nr = n / hs;
+            int sum0 = 0, sum1 = 0, sum2 = 0;
+    #pragma unroll 1
+            for (int r = lane; few && r < nr; r += 32) {
+                const int u = s_P[r * hs + 1] - s_P[r * hs];
+                sum0 += small_div(u + upc - 1, upc);
+                sum1 += small_div(u + upc, upc + 1);
+                sum2 += small_div(u + upc + 1, upc + 2);
+            }
+    #pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) {
+                sum0 += __shfl_xor_sync(0xffffffffu, sum0, sh);
+                sum1 += __shfl_xor_sync(0xffffffffu, sum1, sh);
+                sum2 += __shfl_xor_sync(0xffffffffu, sum2, sh);
+            }
+            const int lim = n_ctas / hs;   // the sums count pieces per head
+            const bool found = few && (sum0 <= lim || sum1 <= lim || sum2 <= lim);
+            const int upc_a = sum0 <= lim ? upc : (sum1 <= lim ? upc + 1 : upc + 2);
+            int carry = 0;
+    #pragma unroll 1
+            for (int base = 0; found && base <= nr; base += 32) {
+                const int r = base + lane;
+                const int v = r < nr ? small_div(s_P[r * hs + 1] - s_P[r * hs] + upc_a - 1, upc_a) : 0;
+                int incl = v;
+    #pragma unroll
+                for (int sh = 1; sh < 32; sh <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, incl, sh);
+                    if (lane >= sh) incl += o;
+                }
+                if (r < nr) {
+    #pragma unroll 1
+                    for (int h = 0; h < hs; ++h) s_Q[r * hs + h] = (carry + incl - v) * hs + h * v;
+                } else if (r == nr) {
+                    s_Q[n] = (carry + incl - v) * hs;
+                }
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) s_aligned = found ? 1 : 0;
+        }
+        __syncthreads();
+        DECODE_TRACE(14);
+        aligned = s_aligned != 0;
+
+        // an item without rows yields zeros - or, when a token is appended, that token's value (softmax over one key)
+        for (int r = blockIdx.x; r < n; r += n_ctas) {
+            if (s_P[r + 1] != s_P[r]) continue;
+            const int reg = r / hs;
+            for (int i = tid; i < p.Hq * D; i += C::THREADS) {
+                float v = 0.f;
+                if (p.k_new) {
+                    const int kvh = HS ? r % hs : (i / D) / p.G;
+                    v = bf16_to_f32(p.v_new[((int64_t)reg * p.kv_heads + kvh) * D + i % D]);
+                }
+                p.out[(int64_t)r * p.Hq * D + i] = v;
+            }
+            if (p.k_new) {
+                const int heads = HS ? 1 : p.kv_heads, h0 = HS ? r % hs : 0;
+                for (int i = tid; i < heads * D; i += C::THREADS) {
+                    const int64_t src = ((int64_t)reg * p.kv_heads + h0) * D + i;
+                    const int64_t dst = ((int64_t)s_off[r] * p.kv_heads + h0) * D + i;
+                    p.k_cache[dst] = p.k_new[src];
+                    p.v_cache[dst] = p.v_new[src];
+                }
+            }
+        }
+        if (aligned) {
+            const int c = (int)blockIdx.x;
+            if (c >= s_Q[n]) { finish(true); return; }
+            const int r = find_region(s_Q, n, c);      // largest r with s_Q[r] <= c: the region this CTA cuts
+            const int pieces = s_Q[r + 1] - s_Q[r], j = c - s_Q[r], units = s_P[r + 1] - s_P[r];
+            u0 = s_P[r] + small_div(units * j, pieces);          // units * pieces < 2^24: both are at most a few thousand
+            u1 = s_P[r] + small_div(units * (j + 1), pieces);
+        } else {
+            u0 = min(total, (int)blockIdx.x * upc);
+            u1 = min(total, u0 + upc);
+        }
     }
     if (u0 >= u1) { finish(true); return; }
     DECODE_TRACE(1);
@@ -343,7 +471,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     if (wid == NCW) {
         // =============================== producer warp ===============================
         if (lane == 0) {
-            int r = find_region(s_P, n, u0);
+            int r = r_own >= 0 ? r_own : find_region(s_P, n, u0);
             int row_base = s_off[r];
             int it = 0;
             bool ok = true;
@@ -612,7 +740,37 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const int items = p.Hq * D / 4;
                 const int np = c1 - c0 + 1;
                 float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)r * p.Hq * D);
-                if (uend == u1 && (size_t)np * slot_floats * 4 <= (size_t)kStages * C::STAGE_BYTES) {
+                if (np == 2) {
+                    // Two pieces: this CTA's half is still in the registers of its ks = 0 warps, so only the
+                    // other half is fetched (one round trip).  Products first, then one addition: the result
+                    // does not depend on which of the two CTAs came last.
+                    if (ks == 0) {
+                        const int other = (int)blockIdx.x == c0 ? c1 : c0;
+                        const float *base = p.partials + (size_t)slot_of(other, r) * slot_floats;
+#pragma unroll
+                        for (int i = 0; i < NROW; ++i) {
+                            const int hl = gid + 8 * i;
+                            if (hl >= G) continue;
+                            const int h = g * G + hl;
+                            const float m2 = __ldcg(base + (size_t)p.Hq * D + h);
+                            const float l2 = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
+                            float2 x[D / 8];
+#pragma unroll
+                            for (int nd = 0; nd < D / 8; ++nd)
+                                x[nd] = __ldcg(reinterpret_cast<const float2 *>(base + (size_t)h * D + nd * 8 + 2 * t));
+                            const float mn = fmaxf(m_run[i], m2);
+                            const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
+                            const float den = __fadd_rn(__fmul_rn(l_run[i], a), __fmul_rn(l2, b));
+                            const float inv = den > 0.f ? 1.0f / den : 0.f;
+                            float *o = p.out + ((int64_t)r * p.Hq + h) * D;
+#pragma unroll
+                            for (int nd = 0; nd < D / 8; ++nd)
+                                *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) = make_float2(
+                                    __fmul_rn(__fadd_rn(__fmul_rn(oacc[nd][2 * i], a), __fmul_rn(x[nd].x, b)), inv),
+                                    __fmul_rn(__fadd_rn(__fmul_rn(oacc[nd][2 * i + 1], a), __fmul_rn(x[nd].y, b)), inv));
+                        }
+                    }
+                } else if (uend == u1 && (size_t)np * slot_floats * 4 <= (size_t)kStages * C::STAGE_BYTES) {
                     // This CTA has no unit left, so the ring is empty: pull all partials of the region into it
                     // with bulk copies (one round trip for everything), then merge out of shared memory.  The
                     // loops below are rolled on purpose: the code runs once and cold instructions cost more
@@ -704,9 +862,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
     };
 
-    int r = find_region(s_P, n, u0);
+    int r = r_own >= 0 ? r_own : find_region(s_P, n, u0);
     int seg_start = u0;
-    len = p.lens[r / hs];
+    len = r_own >= 0 ? len_own : p.lens[r / hs];
     load_q(r);
     int it = 0;
     bool ok = true;
