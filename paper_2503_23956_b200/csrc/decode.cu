@@ -47,11 +47,19 @@ namespace {
         if (threadIdx.x == 0) {                                                                             \
             unsigned long long _t;                                                                          \
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));                                          \
-            reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 16 + (idx)] = _t; \
+            reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 24 + (idx)] = _t; \
         }                                                                                                   \
+    } while (0)
+// the same from whichever thread runs it (the producer lane)
+#define DECODE_TRACE_ANY(idx)                                                                               \
+    do {                                                                                                    \
+        unsigned long long _t;                                                                              \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));                                              \
+        reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 24 + (idx)] = _t; \
     } while (0)
 #else
 #define DECODE_TRACE(idx) do { } while (0)
+#define DECODE_TRACE_ANY(idx) do { } while (0)
 #endif
 
 struct DecodeParams {
@@ -146,6 +154,9 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
     return lo;
 }
 
+// Head-split launches have at least two KV heads per region, so at most kMaxDecodeCtas / 2 regions.
+constexpr int kPlanRegionsPerLane = kMaxDecodeCtas / 2 / 32;
+
 // The region-aligned cut for few regions, planned by one warp in registers (all warps of a CTA call this and
 // get the same answer).  With no more items than CTAs a CTA needs five numbers of the cut: its item, the
 // item's units and rows, its piece and the piece count.  Each lane takes rpl consecutive regions; sums and the
@@ -153,10 +164,10 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
 // the producer can issue its first loads one global round trip after the kernel may read memory.
 // Returns 0 when the tables have to decide (empty regions, too many regions, no fitting cut), 2 when this CTA
 // has no piece, 1 with plan = {item, rows of the item, first unit, end unit} and the item's table entries
-// stored (units counted from the item's first one).
+// stored if `store` is set (units counted from the item's first one).
 __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64_t *offsets, int n, int hs, int n_ctas,
-                                                int ch_log2, int c, int *s_P, int *s_off, int *s_Q, int4 *plan) {
-    constexpr int RPL = kMaxDecodeCtas / 32;
+                                                int ch_log2, int c, bool store, int *s_P, int *s_off, int *s_Q, int4 *plan) {
+    constexpr int RPL = kPlanRegionsPerLane;
     const int lane = threadIdx.x & 31;
     const int nr = n / hs;
     if (n > n_ctas || nr <= 0 || nr > 32 * RPL) return 0;
@@ -187,12 +198,14 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
     const int upc = max(1, small_div(tot * hs + n_ctas - 1, n_ctas));
     // pieces of at most upc_a units: the smallest of upc, upc + 1, upc + 2 that needs no more CTAs than there are
     int sum0 = 0, sum1 = 0, sum2 = 0;
+    int pc0[RPL], pc1[RPL], pc2[RPL];
 #pragma unroll
     for (int j = 0; j < RPL; ++j) {
+        pc0[j] = pc1[j] = pc2[j] = 0;
         if (j < rpl) {
-            sum0 += small_div(un[j] + upc - 1, upc);
-            sum1 += small_div(un[j] + upc, upc + 1);
-            sum2 += small_div(un[j] + upc + 1, upc + 2);
+            sum0 += pc0[j] = small_div(un[j] + upc - 1, upc);
+            sum1 += pc1[j] = small_div(un[j] + upc, upc + 1);
+            sum2 += pc2[j] = small_div(un[j] + upc + 1, upc + 2);
         }
     }
     sum0 = __reduce_add_sync(0xffffffffu, sum0);
@@ -200,12 +213,11 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
     sum2 = __reduce_add_sync(0xffffffffu, sum2);
     const int lim = n_ctas / hs;   // the sums count pieces per head
     if (sum0 > lim && sum1 > lim && sum2 > lim) return 0;
-    const int upc_a = sum0 <= lim ? upc : (sum1 <= lim ? upc + 1 : upc + 2);
     int pc[RPL];
     int mine = 0;
 #pragma unroll
     for (int j = 0; j < RPL; ++j) {
-        pc[j] = j < rpl ? small_div(un[j] + upc_a - 1, upc_a) : 0;
+        pc[j] = sum0 <= lim ? pc0[j] : (sum1 <= lim ? pc1[j] : pc2[j]);
         mine += pc[j];
     }
     int incl = mine;
@@ -236,11 +248,17 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
     v_ln = __shfl_sync(0xffffffffu, v_ln, src);
     v_of = __shfl_sync(0xffffffffu, v_of, src);
     const int rel = c - v_first * hs;
-    const int h = small_div(rel, v_pc), j = rel - h * v_pc;
+    int h = rel, j = 0, first_unit = 0, end_unit = v_un;
+    if (v_pc > 1) {   // (most items are one piece: no division then)
+        h = small_div(rel, v_pc);
+        j = rel - h * v_pc;
+        // no overflow: the units of all regions together are below 2^22, the pieces at most 256
+        first_unit = small_div(v_un * j, v_pc);
+        end_unit = small_div(v_un * (j + 1), v_pc);
+    }
     const int item = v_reg * hs + h;
-    // no overflow: the units of all regions together are below 2^22, the pieces at most 256
-    *plan = make_int4(item, v_ln, small_div(v_un * j, v_pc), small_div(v_un * (j + 1), v_pc));
-    if (lane == 0) {
+    *plan = make_int4(item, v_ln, first_unit, end_unit);
+    if (lane == 0 && store) {
         s_P[item] = 0;
         s_P[item + 1] = v_un;
         s_off[item] = v_of;
@@ -292,9 +310,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s_abort = 0;
     }
+    // made-up region lengths (one unit each) and first rows for the rehearsal of the register plan below
+    constexpr int kPlanRegions = 32 * kPlanRegionsPerLane;
+    int32_t *rehearsal_lens = reinterpret_cast<int32_t *>(s_part);
+    int64_t *rehearsal_offsets = reinterpret_cast<int64_t *>(s_part + kPlanRegions);
+    if (HS && tid < kPlanRegions) { rehearsal_lens[tid] = CH; rehearsal_offsets[tid] = 0; }
     // The barriers are initialised before any warp goes its own way (nothing above read global memory).
     __syncthreads();
-    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     int total = 0, upc = 1;
     bool aligned = false;
@@ -316,14 +338,30 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // ---- few regions: every warp plans for itself, in registers; otherwise the tables below decide ----
     bool planned = false;
     if constexpr (HS) {   // head-split launches are the ones with few items; the by-region kernels keep their registers
+        // The plan runs twice through the same instructions: first on the made-up lengths in shared memory, while
+        // the kernel may not read global memory yet, then on the real ones.  A kernel's first pass through a
+        // stretch of code waits for its instructions line by line, which for this serial stretch costs more than
+        // its arithmetic; the rehearsal moves that wait in front of the dependency wait, where the CTA idles.
         int4 plan;
-        const int rc = plan_few_regions(p.lens, p.offsets, n, hs, n_ctas, C::CH_LOG2, (int)blockIdx.x, s_P, s_off, s_Q,
-                                        &plan);
+        int rc = 0;
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                DECODE_TRACE(16);
+            }
+            rc = plan_few_regions(pass ? p.lens : rehearsal_lens, pass ? p.offsets : rehearsal_offsets, n, hs, n_ctas,
+                                  C::CH_LOG2, (int)blockIdx.x, pass != 0, s_P, s_off, s_Q, &plan);
+        }
         if (rc == 2) { finish(true); return; }
         if (rc == 1) {
             planned = aligned = true;
             r_own = plan.x; len_own = plan.y; u0 = plan.z; u1 = plan.w;
         }
+    }
+    else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        DECODE_TRACE(16);
     }
     DECODE_TRACE(12);
     if (!planned) {
@@ -498,6 +536,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         tma_load_3d(dst + C::KV_BYTES + off, &tm_v, hf * 64, head, row0, full);
                     }
                 }
+                if (it == 0) DECODE_TRACE_ANY(17);
             }
             if (!ok) {
                 // drain: wait (bounded) for the loads already in flight before the CTA may exit
@@ -866,6 +905,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     int seg_start = u0;
     len = r_own >= 0 ? len_own : p.lens[r / hs];
     load_q(r);
+    DECODE_TRACE(18);
     int it = 0;
     bool ok = true;
     for (int u = u0; u < u1; ++u, ++it) {
