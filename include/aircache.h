@@ -243,10 +243,11 @@ int aircache_append(const aircache_shape_t *shape, aircache_ragged_t *cache, con
                     const void *v_new, int32_t appended, void *cuda_stream);
 
 /*
- * Zeroes the status word and the tickets at the start of a workspace (enqueued
- * on the stream).  Must be called once after allocating the workspace, before
- * its first use by aircache_budget or aircache_decode_attn, and again after an
- * AIRCACHE_ERR_TIMEOUT.
+ * Zeroes the head of a workspace (enqueued on the stream): the status word, the
+ * tickets and the plans that decode launches keep from one call to the next
+ * (about 150 KB in all).  Must be called once after allocating the workspace,
+ * before its first use by aircache_budget or aircache_decode_attn, and again
+ * after an AIRCACHE_ERR_TIMEOUT.
  */
 int aircache_reset_status(void *workspace, int64_t workspace_bytes, void *cuda_stream);
 

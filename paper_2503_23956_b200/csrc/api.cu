@@ -62,6 +62,7 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     };
     w.status = take(256);
     w.tickets = take((int64_t)kMaxRegions * 4);
+    w.plan_memo = take(kPlanMemoBytes);
     w.row_count = take(groups * 4);
     w.row_info = take(groups * cap * 4);
     w.row_coef = take(groups * cap * 4);
@@ -262,8 +263,8 @@ int aircache_append(const aircache_shape_t *shape, aircache_ragged_t *cache, con
 int aircache_reset_status(void *workspace, int64_t workspace_bytes, void *cuda_stream) {
     if (!workspace) return AIRCACHE_ERR_INVALID_ARG;
     if ((uintptr_t)workspace & 255) return AIRCACHE_ERR_ALIGNMENT;
-    if (workspace_bytes < kStatusBytes) return AIRCACHE_ERR_WORKSPACE_TOO_SMALL;
-    AIRCACHE_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)cuda_stream));
+    if (workspace_bytes < kResetBytes) return AIRCACHE_ERR_WORKSPACE_TOO_SMALL;
+    AIRCACHE_CUDA_TRY(cudaMemsetAsync(workspace, 0, kResetBytes, (cudaStream_t)cuda_stream));
     return AIRCACHE_OK;
 }
 

@@ -16,6 +16,13 @@ constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode gr
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int64_t kStatusBytes = 256 + (int64_t)kMaxRegions * 4;  // status word + tickets, at the start of the workspace
+// Head-split decode launches (at least two KV heads per region, so at most kMaxDecodeCtas / 2 regions) keep, per
+// CTA, the plan of their last call: 16 words of outcome and the unit count of every region.
+constexpr int kPlanRegionsPerLane = kMaxDecodeCtas / 2 / 32;
+constexpr int kPlanMemoInts = 16 + 32 * kPlanRegionsPerLane;
+constexpr int64_t kPlanMemoBytes = (int64_t)kMaxDecodeCtas * kPlanMemoInts * 4;
+// what aircache_reset_status clears: status word, tickets and the kept plans, which follow them
+constexpr int64_t kResetBytes = kStatusBytes + kPlanMemoBytes;
 
 // ---------------------------------------------------------------------------------------------
 // error plumbing
@@ -83,6 +90,7 @@ inline int score_chunks(const aircache_shape_t *s) {
 struct WsLayout {
     int64_t status;       // u32 status word (256 bytes reserved)
     int64_t tickets;      // i32  [kMaxRegions]        split-K tickets of the decode kernel, zero between calls
+    int64_t plan_memo;    // i32  [kMaxDecodeCtas][kPlanMemoInts]  kept plans of the decode kernel, zero before first use
     int64_t row_count;    // i32  [L*B*Hkv]            elite rows of the KV group
     int64_t row_info;     // i32  [L*B*Hkv][cap]       (head within group << 8) | window slot
     int64_t row_coef;     // f32  [L*B*Hkv][cap]       1 / (|E_h| * Hq)

@@ -65,6 +65,7 @@ namespace {
 struct DecodeParams {
     const uint16_t *q;       // [L*B, Hq, D]
     float *out;              // [L*B, Hq, D]
+    int32_t *plan_memo;    // [kMaxDecodeCtas][kPlanMemoInts] kept plans of the head-split launches, or null
     const int64_t *offsets;  // [L*B + 1]
     const int32_t *lens;     // [L*B]
     int32_t *tickets;        // [L*B] partials of the region written so far; zero between calls
@@ -144,6 +145,14 @@ __device__ __forceinline__ int small_div(int a, int b) {
     return q;
 }
 
+// The same for operands known to be below 2^23: no integer-division fallback to schedule around.
+__device__ __forceinline__ int small_div_unchecked(int a, int b) {
+    int q = (int)__fdividef((float)a, (float)b);
+    if (q * b > a) --q;
+    if ((q + 1) * b <= a) ++q;
+    return q;
+}
+
 // largest r with P[r] <= u (P non-decreasing, P[0] = 0, u < P[n])
 __device__ __forceinline__ int find_region(const int *P, int n, int u) {
     int lo = 0, hi = n - 1;
@@ -154,9 +163,6 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
     return lo;
 }
 
-// Head-split launches have at least two KV heads per region, so at most kMaxDecodeCtas / 2 regions.
-constexpr int kPlanRegionsPerLane = kMaxDecodeCtas / 2 / 32;
-
 // The region-aligned cut for few regions, planned by one warp in registers (all warps of a CTA call this and
 // get the same answer).  With no more items than CTAs a CTA needs five numbers of the cut: its item, the
 // item's units and rows, its piece and the piece count.  Each lane takes rpl consecutive regions; sums and the
@@ -165,25 +171,38 @@ constexpr int kPlanRegionsPerLane = kMaxDecodeCtas / 2 / 32;
 // Returns 0 when the tables have to decide (empty regions, too many regions, no fitting cut), 2 when this CTA
 // has no piece, 1 with plan = {item, rows of the item, first unit, end unit} and the item's table entries
 // stored if `store` is set (units counted from the item's first one).
+//
+// `memo` (may be null) points at this CTA's kPlanMemoInts words of global memory, zero before their first use.
+// The cut depends on the regions' unit counts alone, and those change only every CH appended tokens, so the CTA
+// keeps the unit counts it planned for and the outcome; when the counts read now equal the kept ones, the
+// outcome is taken from there and the arithmetic (about a microsecond of dependent steps) is skipped.  A CTA
+// reads and writes only its own words, and only after the kernel's dependency wait (the rehearsal passes words
+// in shared memory, hence the plain loads).
+//   words 0..4: n, hs, n_ctas, ch_log2, outcome (1 or 2);  8..13: item, first unit, end unit, units, first CTA of the
+//   item, pieces;  14: region;  16..: unit count of every region
 __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64_t *offsets, int n, int hs, int n_ctas,
-                                                int ch_log2, int c, bool store, int *s_P, int *s_off, int *s_Q, int4 *plan) {
+                                                int ch_log2, int c, bool store, int32_t *memo, int *s_P, int *s_off,
+                                                int *s_Q, int4 *plan) {
     constexpr int RPL = kPlanRegionsPerLane;
     const int lane = threadIdx.x & 31;
     const int nr = n / hs;
     if (n > n_ctas || nr <= 0 || nr > 32 * RPL) return 0;
     const int rpl = (nr + 31) >> 5;
-    int un[RPL], ln[RPL], of[RPL];
+    int un[RPL], ln[RPL], of[RPL], kept_un[RPL];
     bool nonempty = true;
     int tot = 0;
+    int memo_word = 0;
 #pragma unroll
     for (int j = 0; j < RPL; ++j) {
-        un[j] = ln[j] = of[j] = 0;
+        un[j] = ln[j] = of[j] = kept_un[j] = 0;
         const int reg = lane * rpl + j;
         if (j < rpl && reg < nr) {
             ln[j] = max(lens[reg], 0);
             of[j] = (int)offsets[reg];
+            if (memo) kept_un[j] = memo[16 + reg];
         }
     }
+    if (memo && lane < 16) memo_word = memo[lane];
 #pragma unroll
     for (int j = 0; j < RPL; ++j) {
         const int reg = lane * rpl + j;
@@ -193,19 +212,63 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
             tot += un[j];
         }
     }
+    if (memo) {
+        const int expect = lane == 0 ? n : (lane == 1 ? hs : (lane == 2 ? n_ctas : ch_log2));
+        bool same = lane >= 4 || memo_word == expect;
+        if (lane == 4) same = memo_word == 1 || memo_word == 2;
+#pragma unroll
+        for (int j = 0; j < RPL; ++j) same = same && kept_un[j] == un[j];   // (both zero past the last region)
+        if (__all_sync(0xffffffffu, same)) {
+            if (__shfl_sync(0xffffffffu, memo_word, 4) == 2) return 2;
+            const int item = __shfl_sync(0xffffffffu, memo_word, 8);
+            const int first_unit = __shfl_sync(0xffffffffu, memo_word, 9);
+            const int end_unit = __shfl_sync(0xffffffffu, memo_word, 10);
+            const int units = __shfl_sync(0xffffffffu, memo_word, 11);
+            const int q_first = __shfl_sync(0xffffffffu, memo_word, 12);
+            const int pieces = __shfl_sync(0xffffffffu, memo_word, 13);
+            const int reg = __shfl_sync(0xffffffffu, memo_word, 14);
+            // rows and first row of that region as read now: they change with every appended token
+            const int src = small_div_unchecked(reg, rpl), slot = reg - src * rpl;
+            int rows = 0, first_row = 0;
+#pragma unroll
+            for (int j = 0; j < RPL; ++j)
+                if (j == slot) { rows = ln[j]; first_row = of[j]; }
+            rows = __shfl_sync(0xffffffffu, rows, src);
+            first_row = __shfl_sync(0xffffffffu, first_row, src);
+            *plan = make_int4(item, rows, first_unit, end_unit);
+            if (lane == 0 && store) {
+                s_P[item] = 0;
+                s_P[item + 1] = units;
+                s_off[item] = first_row;
+                s_Q[item] = q_first;
+                s_Q[item + 1] = q_first + pieces;
+            }
+            __syncwarp();
+            return 1;
+        }
+    }
+    // one warp of the CTA records what is planned below
+    const bool record = memo != nullptr && store && threadIdx.x < 32;
     tot = __reduce_add_sync(0xffffffffu, tot);   // units of one head's items
+    // (the bound keeps every dividend below 2^23 and units * pieces below 2^31)
     if (!__all_sync(0xffffffffu, nonempty) || tot >= (1 << 22) / hs) return 0;
-    const int upc = max(1, small_div(tot * hs + n_ctas - 1, n_ctas));
-    // pieces of at most upc_a units: the smallest of upc, upc + 1, upc + 2 that needs no more CTAs than there are
+    const int upc = max(1, small_div_unchecked(tot * hs + n_ctas - 1, n_ctas));
+    // An item of at most `cap` units stays whole; a longer one is cut into pieces of at most cap - kSplitCost
+    // units, because its CTAs also publish and merge partials, which takes them about as long as that many
+    // units: the whole items then end the kernel, not the pieces.  Tried in turn: cap = upc + 1, upc + 2, and
+    // upc + 2 with plain pieces of at most cap units (the one that needs the fewest CTAs).
+    constexpr int kSplitCost = 2;
+    const int cap0 = upc + 1, cap1 = upc + 2;
+    const int cut0 = max(1, cap0 - kSplitCost), cut1 = max(1, cap1 - kSplitCost);
     int sum0 = 0, sum1 = 0, sum2 = 0;
     int pc0[RPL], pc1[RPL], pc2[RPL];
 #pragma unroll
     for (int j = 0; j < RPL; ++j) {
         pc0[j] = pc1[j] = pc2[j] = 0;
         if (j < rpl) {
-            sum0 += pc0[j] = small_div(un[j] + upc - 1, upc);
-            sum1 += pc1[j] = small_div(un[j] + upc, upc + 1);
-            sum2 += pc2[j] = small_div(un[j] + upc + 1, upc + 2);
+            sum0 += pc0[j] = un[j] <= cap0 ? 1 : small_div_unchecked(un[j] + cut0 - 1, cut0);
+            sum1 += pc1[j] = un[j] <= cap1 ? 1 : small_div_unchecked(un[j] + cut1 - 1, cut1);
+            sum2 += pc2[j] = small_div_unchecked(un[j] + cap1 - 1, cap1);
         }
     }
     sum0 = __reduce_add_sync(0xffffffffu, sum0);
@@ -239,7 +302,15 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
         }
     }
     const unsigned ball = __ballot_sync(0xffffffffu, v_reg >= 0);
-    if (ball == 0) return 2;   // more CTAs than pieces
+    if (record) {
+#pragma unroll
+        for (int j = 0; j < RPL; ++j)
+            if (j < rpl && lane * rpl + j < nr) __stcg(memo + 16 + lane * rpl + j, un[j]);
+    }
+    if (ball == 0) {   // more CTAs than pieces
+        if (record && lane < 5) __stcg(memo + lane, lane == 0 ? n : (lane == 1 ? hs : (lane == 2 ? n_ctas : (lane == 3 ? ch_log2 : 2))));
+        return 2;
+    }
     const int src = __ffs(ball) - 1;
     v_reg = __shfl_sync(0xffffffffu, v_reg, src);
     v_first = __shfl_sync(0xffffffffu, v_first, src);
@@ -250,7 +321,7 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
     const int rel = c - v_first * hs;
     int h = rel, j = 0, first_unit = 0, end_unit = v_un;
     if (v_pc > 1) {   // (most items are one piece: no division then)
-        h = small_div(rel, v_pc);
+        h = small_div_unchecked(rel, v_pc);
         j = rel - h * v_pc;
         // no overflow: the units of all regions together are below 2^22, the pieces at most 256
         first_unit = small_div(v_un * j, v_pc);
@@ -264,6 +335,16 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
         s_off[item] = v_of;
         s_Q[item] = v_first * hs + h * v_pc;
         s_Q[item + 1] = v_first * hs + (h + 1) * v_pc;
+    }
+    if (record && lane < 16) {
+        const int head[5] = {n, hs, n_ctas, ch_log2, 1};
+        const int body[7] = {item, first_unit, end_unit, v_un, v_first * hs + h * v_pc, v_pc, v_reg};
+        int w = 0;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) if (lane == i) w = head[i];
+#pragma unroll
+        for (int i = 0; i < 7; ++i) if (lane == 8 + i) w = body[i];
+        __stcg(memo + lane, w);
     }
     __syncwarp();
     return 1;
@@ -314,7 +395,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     constexpr int kPlanRegions = 32 * kPlanRegionsPerLane;
     int32_t *rehearsal_lens = reinterpret_cast<int32_t *>(s_part);
     int64_t *rehearsal_offsets = reinterpret_cast<int64_t *>(s_part + kPlanRegions);
-    if (HS && tid < kPlanRegions) { rehearsal_lens[tid] = CH; rehearsal_offsets[tid] = 0; }
+    int32_t *rehearsal_memo = reinterpret_cast<int32_t *>(s_part + 3 * kPlanRegions);   // a kept plan that matches them
+    if (HS && tid < kPlanRegions) {
+        rehearsal_lens[tid] = CH;
+        rehearsal_offsets[tid] = 0;
+        rehearsal_memo[16 + tid] = tid < n / hs ? 1 : 0;
+        if (tid < 16) {
+            // n, hs, n_ctas, log2 CH, outcome 1 | item 0 = units [0, 1) of 1, first CTA 0, one piece, region 0
+            const int words[16] = {n, hs, n_ctas, C::CH_LOG2, 1, 0, 0, 0, 0, 0, 1, 1, 0, 1, 0, 0};
+            int w = 0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) if (tid == i) w = words[i];
+            rehearsal_memo[tid] = w;
+        }
+    }
     // The barriers are initialised before any warp goes its own way (nothing above read global memory).
     __syncthreads();
 
@@ -338,8 +432,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // ---- few regions: every warp plans for itself, in registers; otherwise the tables below decide ----
     bool planned = false;
     if constexpr (HS) {   // head-split launches are the ones with few items; the by-region kernels keep their registers
-        // The plan runs twice through the same instructions: first on the made-up lengths in shared memory, while
-        // the kernel may not read global memory yet, then on the real ones.  A kernel's first pass through a
+        // The plan runs twice through the same instructions: first on the made-up lengths in shared memory (with a
+        // kept plan that matches them, the usual case), while the kernel may not read global memory yet, then on
+        // the real ones.  A kernel's first pass through a
         // stretch of code waits for its instructions line by line, which for this serial stretch costs more than
         // its arithmetic; the rehearsal moves that wait in front of the dependency wait, where the CTA idles.
         int4 plan;
@@ -351,7 +446,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 DECODE_TRACE(16);
             }
             rc = plan_few_regions(pass ? p.lens : rehearsal_lens, pass ? p.offsets : rehearsal_offsets, n, hs, n_ctas,
-                                  C::CH_LOG2, (int)blockIdx.x, pass != 0, s_P, s_off, s_Q, &plan);
+                                  C::CH_LOG2, (int)blockIdx.x, pass != 0,
+                                  !p.plan_memo ? nullptr
+                                               : (pass ? p.plan_memo + (size_t)blockIdx.x * kPlanMemoInts : rehearsal_memo),
+                                  s_P, s_off, s_Q, &plan);
         }
         if (rc == 2) { finish(true); return; }
         if (rc == 1) {
@@ -1035,6 +1133,7 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.offsets = c->offsets;
     p.lens = c->lens;
     p.tickets = ws_ptr<int32_t>(ws, w.tickets);
+    p.plan_memo = ws_ptr<int32_t>(ws, w.plan_memo);
     p.partials = ws_ptr<float>(ws, w.partials);
     p.status = ws_ptr<uint32_t>(ws, w.status);
     p.k_new = (const uint16_t *)k_new;
@@ -1094,6 +1193,7 @@ int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, 
     p.offsets = c->offsets;
     p.lens = c->lens;
     p.status = reinterpret_cast<uint32_t *>(base);
+    p.plan_memo = nullptr;   // the built-in array keeps no plans: every call plans afresh
     p.k_new = p.v_new = nullptr;
     p.k_cache = p.v_cache = nullptr;
     p.lens_rw = nullptr;

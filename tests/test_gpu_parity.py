@@ -404,6 +404,45 @@ def test_fused_decode_step_appends_and_attends(oracle, case):
                                    check=False) == ac.ERR_CAPACITY
 
 
+@pytest.mark.parametrize("case", ["s7b", "s72b", "kv2"])
+def test_decode_plan_kept_between_calls(oracle, case):
+    """Head-split launches keep their plan in the workspace and reuse it while the regions' unit counts stay the
+    same.  The rows in use must still be read afresh: a region one row shorter (same unit count, plan reused), a
+    region cut to a few rows (other unit count, plan redone) and the original lengths again, all on one workspace."""
+    wl = CASES[case]
+    ref = oracle_path(oracle, wl)
+    cp = ref["compact"]
+    gp = make_gpu(wl, ref)
+    run_chain(gp, ref)
+    q = decode_queries(wl, 0, "cpu")
+    qd = q.to(DEV)
+
+    def both(lens):
+        gp.lens.copy_(torch.from_numpy(lens).to(DEV))
+        want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], lens, u16(q), wl.scale)
+        gp.out.fill_(float("nan"))
+        gp.decode(qd)
+        assert gp.status() == 0
+        got = gp.out.cpu().numpy().copy()
+        assert rel_row_err(got, want) <= TOL
+        return got
+
+    lens0 = cp["lens"].copy()
+    first = both(lens0)
+    again = both(lens0)                     # the kept plan
+    assert np.array_equal(first, again)
+    lens1 = lens0.copy()
+    lens1[1] -= 1                           # same units (unless the length was 1 mod the unit): fresh row count
+    both(lens1)
+    lens2 = lens1.copy()
+    lens2[0] = 5                            # one unit instead of several
+    lens2[-1] = max(1, lens2[-1] // 2)
+    both(lens2)
+    both(lens2)
+    back = both(lens0)
+    assert np.array_equal(first, back)
+
+
 def _random_workload(seed):
     rng = np.random.default_rng(1000 + seed)
     hkv = int(rng.choice([1, 2, 4, 8]))
