@@ -63,7 +63,7 @@ extern "C" {
 /* Problem shape, uniform over the batch. */
 typedef struct {
     int32_t n_layers;    /* L >= 1                                                                   */
-    int32_t batch;       /* B >= 1; L * B <= 1920                                                    */
+    int32_t batch;       /* B >= 1; L * B <= 1792                                                    */
     int32_t n_q_heads;   /* Hq, a multiple of n_kv_heads with Hq / Hkv <= 16                         */
     int32_t n_kv_heads;  /* Hkv in {1, 2, 4, 8}                                                      */
     int32_t head_dim;    /* d in {64, 128}                                                           */

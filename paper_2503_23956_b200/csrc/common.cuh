@@ -11,7 +11,7 @@ namespace aircache {
 
 constexpr int kMaxWindow = 64;
 constexpr int kMaxGroup = 16;         // query heads per KV head
-constexpr int kMaxRegions = 1920;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
+constexpr int kMaxRegions = 1792;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
 constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;

@@ -88,6 +88,12 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
+// transposes an 8x8 matrix of 16-bit elements held one row (two elements per thread) per four lanes
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -117,7 +123,7 @@ struct DecodeCfg {
     static constexpr int SUBTILE = CH * 128;         // bytes of one (head, half) box
     static constexpr int KV_BYTES = HKV * HALVES * SUBTILE;
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
-    static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 2));
+    static constexpr int MERGE_FLOATS_PER_WARP = 32 * (NROW * (D / 4 + 4));
     static constexpr int MERGE_SLOTS = KSPLIT / 2;     // tree merge: the upper half of the warps hands over to the lower
     static constexpr int MERGE_BYTES = HKV * MERGE_SLOTS * MERGE_FLOATS_PER_WARP * 4;
     // the prologue's scan scratch lives in the same bytes as the merge buffer (used before the first flush)
@@ -125,8 +131,10 @@ struct DecodeCfg {
     static constexpr int MERGE_STAGE_BYTES = 16384;            // weights [partials][Hq] of the final merge
     static constexpr int SCRATCH_MIN = SCAN_BYTES > MERGE_STAGE_BYTES ? SCAN_BYTES : MERGE_STAGE_BYTES;
     static constexpr int SCRATCH_BYTES = ((MERGE_BYTES > SCRATCH_MIN ? MERGE_BYTES : SCRATCH_MIN) + 15) / 16 * 16;
-    static constexpr int PLAN_BYTES = (kMaxRegions + 2) * 4;   // unit prefix
-    static constexpr int OFFS_BYTES = kMaxRegions * 4;         // first row of every region
+    // (head-split launches have at most kMaxDecodeCtas items)
+    static constexpr int TABLE_ENTRIES = HS ? kMaxDecodeCtas : kMaxRegions;
+    static constexpr int PLAN_BYTES = (TABLE_ENTRIES + 2) * 4;   // unit prefix
+    static constexpr int OFFS_BYTES = TABLE_ENTRIES * 4;         // first row of every region
     // ring depth: what fits beside the scratch and the tables in the 227 KB a CTA may use (1.5 KB are left
     // for static shared memory, 1 KB for the alignment slack), at most 4 stages
     static constexpr int FIT = (232448 - 1536 - 1024 - SCRATCH_BYTES - PLAN_BYTES - OFFS_BYTES - 256) / STAGE_BYTES;
@@ -654,25 +662,31 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     int n_flush = 0;  // flushes done so far (trace slots only)
     int len = 0;      // rows of the item being processed
-    uint32_t qa[D / 16][4];
-    float oacc[D / 8][4];
-    float m_run[2], l_run[2];
+    // The block's products are taken transposed - S^T = K Q^T and O^T = V^T P^T - so that the 16 rows of the tensor
+    // core tile are keys (respectively channels) and its 8 columns the query heads of the KV group: a group of up
+    // to 8 heads fills one column tile, where heads as rows would leave half of a 16-row tile empty.
+    // A thread holds, per column tile nt: heads nt*8 + 2t, +1 of keys gid, gid+8 (S^T) or of channels
+    // mt*16 + gid, +8 (O^T).
+    uint32_t qb[NROW][D / 16][2];     // Q^T as the right-hand operand: head nt*8 + gid, channels kk*16 + 2t.., +8
+    float oacc[NROW][D / 16][4];
+    float m_run[NROW][2], l_run[NROW][2];   // per head 2t, 2t+1; l_run is this thread's share until the flush
 
     auto load_q = [&](int r) {
-        const uint16_t *q_lo = p.q + ((int64_t)r * p.Hq + g * G + gid) * D;
-        const uint16_t *q_hi = q_lo + 8 * D;
-        const bool v_lo = gid < G, v_hi = G_HI && (gid + 8 < G);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-            qa[kk][0] = v_lo ? __ldg(reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 2 * t)) : 0u;
-            qa[kk][2] = v_lo ? __ldg(reinterpret_cast<const uint32_t *>(q_lo + kk * 16 + 8 + 2 * t)) : 0u;
-            qa[kk][1] = v_hi ? __ldg(reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 2 * t)) : 0u;
-            qa[kk][3] = v_hi ? __ldg(reinterpret_cast<const uint32_t *>(q_hi + kk * 16 + 8 + 2 * t)) : 0u;
+        for (int nt = 0; nt < NROW; ++nt) {
+            const int hl = nt * 8 + gid;
+            const bool valid = hl < G;
+            const uint16_t *qp = p.q + ((int64_t)r * p.Hq + g * G + (valid ? hl : 0)) * D;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                qb[nt][kk][0] = valid ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16 + 2 * t)) : 0u;
+                qb[nt][kk][1] = valid ? __ldg(reinterpret_cast<const uint32_t *>(qp + kk * 16 + 8 + 2 * t)) : 0u;
+            }
+#pragma unroll
+            for (int mt = 0; mt < D / 16; ++mt) oacc[nt][mt][0] = oacc[nt][mt][1] = oacc[nt][mt][2] = oacc[nt][mt][3] = 0.f;
+            m_run[nt][0] = m_run[nt][1] = -INFINITY;
+            l_run[nt][0] = l_run[nt][1] = 0.f;
         }
-#pragma unroll
-        for (int nd = 0; nd < D / 8; ++nd) oacc[nd][0] = oacc[nd][1] = oacc[nd][2] = oacc[nd][3] = 0.f;
-        m_run[0] = m_run[1] = -INFINITY;
-        l_run[0] = l_run[1] = 0.f;
     };
 
     // One block of 16 keys at rows blk_row0.. of a (K, V) tile in shared memory; the block's first key is row j0
@@ -680,60 +694,72 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     auto process_block = [&](uint32_t k_base, uint32_t v_base, uint32_t sub_stride, int blk_row0, int j0, int len) {
         const int mi = lane >> 3, rr = lane & 7;
 
-        // ---- S = Q K^T for 16 keys ----
-        float sacc[2][4];
+        // ---- S^T = K Q^T for 16 keys; two accumulators per tile halve the chain of dependent MMAs ----
+        float sacc[NROW][2][4];
 #pragma unroll
-        for (int a = 0; a < 2; ++a) sacc[a][0] = sacc[a][1] = sacc[a][2] = sacc[a][3] = 0.f;
+        for (int nt = 0; nt < NROW; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) sacc[nt][e][0] = sacc[nt][e][1] = sacc[nt][e][2] = sacc[nt][e][3] = 0.f;
         {
-            const int row = blk_row0 + (mi >> 1) * 8 + rr;
+            const int row = blk_row0 + (mi & 1) * 8 + rr;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-                const int hf = kk >> 2, chunk = ((kk & 3) << 1) + (mi & 1);
-                uint32_t b[4];
-                ldmatrix_x4(b, k_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
-                mma_bf16_16816(sacc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[0], b[1]);
-                mma_bf16_16816(sacc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b[2], b[3]);
+                const int hf = kk >> 2, chunk = ((kk & 3) << 1) + (mi >> 1);
+                uint32_t a[4];   // keys 0-7 / 8-15 of channels kk*16.., then of channels kk*16 + 8..
+                ldmatrix_x4(a, k_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
+#pragma unroll
+                for (int nt = 0; nt < NROW; ++nt)
+                    mma_bf16_16816(sacc[nt][kk & 1], a[0], a[1], a[2], a[3], qb[nt][kk][0], qb[nt][kk][1]);
             }
         }
         // ---- online softmax (exp2 domain) ----
         const bool tail = j0 + 16 > len;
-        uint32_t pa[4], pb[4];  // P = pa + pb: bf16 head and bf16 remainder of every probability
-        float corr[2];
+        const bool dead_lo = tail && j0 + gid >= len, dead_hi = tail && j0 + gid + 8 >= len;
+        uint32_t pa[NROW][2], pb[NROW][2];  // P^T = pa + pb (bf16 head and bf16 remainder), as right-hand operands
+        bool rescale = false;
+        float corr[NROW][2];
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            if (i >= NROW) { pa[i] = pa[i + 2] = pb[i] = pb[i + 2] = 0u; corr[i] = 1.f; continue; }
-            float x[4];
-            x[0] = sacc[0][2 * i] * p.sl2; x[1] = sacc[0][2 * i + 1] * p.sl2;
-            x[2] = sacc[1][2 * i] * p.sl2; x[3] = sacc[1][2 * i + 1] * p.sl2;
-            if (tail) {
-                const int jk = j0 + 2 * t;
-                if (jk >= len) x[0] = -INFINITY;
-                if (jk + 1 >= len) x[1] = -INFINITY;
-                if (jk + 8 >= len) x[2] = -INFINITY;
-                if (jk + 9 >= len) x[3] = -INFINITY;
-            }
-            float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float mn = fmaxf(m_run[i], mx);  // finite: row j0 of the block is valid
-            corr[i] = exp2_or_zero(m_run[i], mn);
-            m_run[i] = mn;
-            const float e0 = fast_exp2(x[0] - mn), e1 = fast_exp2(x[1] - mn);
-            const float e2 = fast_exp2(x[2] - mn), e3 = fast_exp2(x[3] - mn);
-            pa[i] = pack_bf16(e0, e1);
-            pa[i + 2] = pack_bf16(e2, e3);
-            pb[i] = pack_bf16(e0 - bf16lo(pa[i]), e1 - bf16hi(pa[i]));
-            pb[i + 2] = pack_bf16(e2 - bf16lo(pa[i + 2]), e3 - bf16hi(pa[i + 2]));
-            l_run[i] = l_run[i] * corr[i] + ((e0 + e1) + (e2 + e3));
-        }
-        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+        for (int nt = 0; nt < NROW; ++nt) {
+            float x[4];   // keys gid (heads 2t, 2t+1), gid + 8 (heads 2t, 2t+1)
 #pragma unroll
-            for (int nd = 0; nd < D / 8; ++nd) {
-                oacc[nd][0] *= corr[0]; oacc[nd][1] *= corr[0];
-                if (G_HI) { oacc[nd][2] *= corr[1]; oacc[nd][3] *= corr[1]; }
+            for (int i = 0; i < 4; ++i) x[i] = (sacc[nt][0][i] + sacc[nt][1][i]) * p.sl2;
+            if (dead_lo) x[0] = x[1] = -INFINITY;
+            if (dead_hi) x[2] = x[3] = -INFINITY;
+            float mx0 = fmaxf(x[0], x[2]), mx1 = fmaxf(x[1], x[3]);
+#pragma unroll
+            for (int sh = 4; sh < 32; sh <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
             }
+            const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);  // finite: key j0 is valid
+            corr[nt][0] = exp2_or_zero(m_run[nt][0], mn0);
+            corr[nt][1] = exp2_or_zero(m_run[nt][1], mn1);
+            rescale = rescale || corr[nt][0] != 1.f || corr[nt][1] != 1.f;
+            m_run[nt][0] = mn0;
+            m_run[nt][1] = mn1;
+            const float e0 = fast_exp2(x[0] - mn0), e1 = fast_exp2(x[1] - mn1);
+            const float e2 = fast_exp2(x[2] - mn0), e3 = fast_exp2(x[3] - mn1);
+            const uint32_t a_lo = pack_bf16(e0, e1), a_hi = pack_bf16(e2, e3);   // key gid, key gid + 8
+            const uint32_t b_lo = pack_bf16(e0 - bf16lo(a_lo), e1 - bf16hi(a_lo));
+            const uint32_t b_hi = pack_bf16(e2 - bf16lo(a_hi), e3 - bf16hi(a_hi));
+            l_run[nt][0] = l_run[nt][0] * corr[nt][0] + (e0 + e2);
+            l_run[nt][1] = l_run[nt][1] * corr[nt][1] + (e1 + e3);
+            // (key gid; heads 2t, 2t+1) -> (keys 2t, 2t+1; head gid): the operand layout of the second product
+            pa[nt][0] = movmatrix_trans(a_lo);
+            pa[nt][1] = movmatrix_trans(a_hi);
+            pb[nt][0] = movmatrix_trans(b_lo);
+            pb[nt][1] = movmatrix_trans(b_hi);
         }
-        // ---- O += P V ----
+        if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+            for (int nt = 0; nt < NROW; ++nt)
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) {
+                    oacc[nt][mt][0] *= corr[nt][0]; oacc[nt][mt][1] *= corr[nt][1];
+                    oacc[nt][mt][2] *= corr[nt][0]; oacc[nt][mt][3] *= corr[nt][1];
+                }
+        }
+        // ---- O^T += V^T P^T ----
         uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
         if (tail) {
             // rows past the region's end may hold anything (slack is never written): clear them so that
@@ -743,18 +769,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             vmask1 = (jk + 8 < len ? 0x0000ffffu : 0u) | (jk + 9 < len ? 0xffff0000u : 0u);
         }
         {
-            const int row = blk_row0 + (mi & 1) * 8 + rr;
+            const int row = blk_row0 + (mi >> 1) * 8 + rr;
 #pragma unroll
-            for (int n2 = 0; n2 < D / 16; ++n2) {
-                const int cg = n2 * 2 + (mi >> 1);
+            for (int mt = 0; mt < D / 16; ++mt) {
+                const int cg = mt * 2 + (mi & 1);
                 const int hf = cg >> 3, chunk = cg & 7;
-                uint32_t b[4];
-                ldmatrix_x4_trans(b, v_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
-                if (tail) { b[0] &= vmask0; b[1] &= vmask1; b[2] &= vmask0; b[3] &= vmask1; }
-                mma_bf16_16816(oacc[2 * n2], pa[0], pa[1], pa[2], pa[3], b[0], b[1]);
-                mma_bf16_16816(oacc[2 * n2 + 1], pa[0], pa[1], pa[2], pa[3], b[2], b[3]);
-                mma_bf16_16816(oacc[2 * n2], pb[0], pb[1], pb[2], pb[3], b[0], b[1]);
-                mma_bf16_16816(oacc[2 * n2 + 1], pb[0], pb[1], pb[2], pb[3], b[2], b[3]);
+                uint32_t a[4];   // channels mt*16.. / +8 of keys 2t, 2t+1, then of keys 2t+8, 2t+9
+                ldmatrix_x4_trans(a, v_base + hf * sub_stride + row * 128 + ((chunk ^ (row & 7)) << 4));
+                if (tail) { a[0] &= vmask0; a[1] &= vmask0; a[2] &= vmask1; a[3] &= vmask1; }
+#pragma unroll
+                for (int nt = 0; nt < NROW; ++nt) {
+                    mma_bf16_16816(oacc[nt][mt], a[0], a[1], a[2], a[3], pa[nt][0], pa[nt][1]);
+                    mma_bf16_16816(oacc[nt][mt], a[0], a[1], a[2], a[3], pb[nt][0], pb[nt][1]);
+                }
             }
         }
     };
@@ -785,10 +812,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             consumer_bar(NCW * 32);   // the scratch area becomes the merge buffer below
         }
 #pragma unroll
-        for (int i = 0; i < NROW; ++i) {
-            l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
-            l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
-        }
+        for (int nt = 0; nt < NROW; ++nt)
+#pragma unroll
+            for (int sh = 4; sh < 32; sh <<= 1) {
+                l_run[nt][0] += __shfl_xor_sync(0xffffffffu, l_run[nt][0], sh);
+                l_run[nt][1] += __shfl_xor_sync(0xffffffffu, l_run[nt][1], sh);
+            }
         // the KSPLIT warps of a KV head merge their states pairwise: in every round the upper half of the
         // remaining warps hands its (max, sum, accumulator) to the lower half through shared memory
 #pragma unroll
@@ -797,14 +826,15 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 float *dst = s_merge + (size_t)(g * C::MERGE_SLOTS + ks - half) * C::MERGE_FLOATS_PER_WARP + lane;
                 int c = 0;
 #pragma unroll
-                for (int i = 0; i < NROW; ++i) {
-                    dst[32 * c++] = m_run[i];
-                    dst[32 * c++] = l_run[i];
+                for (int nt = 0; nt < NROW; ++nt) {
+                    dst[32 * c++] = m_run[nt][0];
+                    dst[32 * c++] = m_run[nt][1];
+                    dst[32 * c++] = l_run[nt][0];
+                    dst[32 * c++] = l_run[nt][1];
 #pragma unroll
-                    for (int nd = 0; nd < D / 8; ++nd) {
-                        dst[32 * c++] = oacc[nd][2 * i];
-                        dst[32 * c++] = oacc[nd][2 * i + 1];
-                    }
+                    for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) dst[32 * c++] = oacc[nt][mt][i];
                 }
             }
             consumer_bar(NCW * 32);
@@ -812,50 +842,62 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const float *src = s_merge + (size_t)(g * C::MERGE_SLOTS + ks) * C::MERGE_FLOATS_PER_WARP + lane;
                 int c = 0;
 #pragma unroll
-                for (int i = 0; i < NROW; ++i) {
-                    const float m2 = src[32 * c++];
-                    const float l2 = src[32 * c++];
-                    const float mn = fmaxf(m_run[i], m2);
-                    const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
-                    l_run[i] = l_run[i] * a + l2 * b;
-                    m_run[i] = mn;
+                for (int nt = 0; nt < NROW; ++nt) {
+                    float a[2], b[2];
+                    const float m2[2] = {src[32 * c], src[32 * (c + 1)]};
+                    const float l2[2] = {src[32 * (c + 2)], src[32 * (c + 3)]};
+                    c += 4;
 #pragma unroll
-                    for (int nd = 0; nd < D / 8; ++nd) {
-                        oacc[nd][2 * i] = oacc[nd][2 * i] * a + src[32 * c++] * b;
-                        oacc[nd][2 * i + 1] = oacc[nd][2 * i + 1] * a + src[32 * c++] * b;
+                    for (int e = 0; e < 2; ++e) {
+                        const float mn = fmaxf(m_run[nt][e], m2[e]);
+                        a[e] = exp2_or_zero(m_run[nt][e], mn);
+                        b[e] = exp2_or_zero(m2[e], mn);
+                        l_run[nt][e] = l_run[nt][e] * a[e] + l2[e] * b[e];
+                        m_run[nt][e] = mn;
                     }
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            oacc[nt][mt][i] = oacc[nt][mt][i] * a[i & 1] + src[32 * c++] * b[i & 1];
                 }
             }
             consumer_bar(NCW * 32);
         }
         const bool whole = (ustart == s_P[r]) && (uend == s_P[r + 1]);
         if (ks == 0) {
+            // this thread's values: heads nt*8 + 2t + e, channels mt*16 + gid and + 8 (the eight gid lanes of a
+            // store instruction cover 32 consecutive bytes of a head's row)
 #pragma unroll
-            for (int i = 0; i < NROW; ++i) {
-                const int hl = gid + 8 * i;
-                if (hl >= G) continue;
-                const int h = g * G + hl;
-                if (whole) {
-                    const float inv = l_run[i] > 0.f ? 1.0f / l_run[i] : 0.f;
-                    float *o = p.out + ((int64_t)r * p.Hq + h) * D;
+            for (int nt = 0; nt < NROW; ++nt)
 #pragma unroll
-                    for (int nd = 0; nd < D / 8; ++nd)
-                        *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) =
-                            make_float2(oacc[nd][2 * i] * inv, oacc[nd][2 * i + 1] * inv);
-                } else {
-                    const int slot = slot_of((int)blockIdx.x, r);
-                    float *base = p.partials + (size_t)slot * partial_slot_floats(p.Hq, D);
-                    float *o = base + (size_t)h * D;
+                for (int e = 0; e < 2; ++e) {
+                    const int hl = nt * 8 + 2 * t + e;
+                    if (hl >= G) continue;
+                    const int h = g * G + hl;
+                    if (whole) {
+                        const float inv = l_run[nt][e] > 0.f ? 1.0f / l_run[nt][e] : 0.f;
+                        float *o = p.out + ((int64_t)r * p.Hq + h) * D + gid;
 #pragma unroll
-                    for (int nd = 0; nd < D / 8; ++nd)
-                        __stcg(reinterpret_cast<float2 *>(o + nd * 8 + 2 * t),
-                               make_float2(oacc[nd][2 * i], oacc[nd][2 * i + 1]));
-                    if (t == 0) {
-                        __stcg(base + (size_t)p.Hq * D + h, m_run[i]);
-                        __stcg(base + (size_t)p.Hq * (D + 1) + h, l_run[i]);
+                        for (int mt = 0; mt < D / 16; ++mt) {
+                            o[mt * 16] = oacc[nt][mt][e] * inv;
+                            o[mt * 16 + 8] = oacc[nt][mt][2 + e] * inv;
+                        }
+                    } else {
+                        const int slot = slot_of((int)blockIdx.x, r);
+                        float *base = p.partials + (size_t)slot * partial_slot_floats(p.Hq, D);
+                        float *o = base + (size_t)h * D + gid;
+#pragma unroll
+                        for (int mt = 0; mt < D / 16; ++mt) {
+                            __stcg(o + mt * 16, oacc[nt][mt][e]);
+                            __stcg(o + mt * 16 + 8, oacc[nt][mt][2 + e]);
+                        }
+                        if (gid == 0) {
+                            __stcg(base + (size_t)p.Hq * D + h, m_run[nt][e]);
+                            __stcg(base + (size_t)p.Hq * (D + 1) + h, l_run[nt][e]);
+                        }
                     }
                 }
-            }
         }
         if (!whole) {
             // split-K combine without a second launch: publish the partial, draw a ticket; the CTA that draws
@@ -885,27 +927,33 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         const int other = (int)blockIdx.x == c0 ? c1 : c0;
                         const float *base = p.partials + (size_t)slot_of(other, r) * slot_floats;
 #pragma unroll
-                        for (int i = 0; i < NROW; ++i) {
-                            const int hl = gid + 8 * i;
-                            if (hl >= G) continue;
-                            const int h = g * G + hl;
-                            const float m2 = __ldcg(base + (size_t)p.Hq * D + h);
-                            const float l2 = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
-                            float2 x[D / 8];
+                        for (int nt = 0; nt < NROW; ++nt)
 #pragma unroll
-                            for (int nd = 0; nd < D / 8; ++nd)
-                                x[nd] = __ldcg(reinterpret_cast<const float2 *>(base + (size_t)h * D + nd * 8 + 2 * t));
-                            const float mn = fmaxf(m_run[i], m2);
-                            const float a = exp2_or_zero(m_run[i], mn), b = exp2_or_zero(m2, mn);
-                            const float den = __fadd_rn(__fmul_rn(l_run[i], a), __fmul_rn(l2, b));
-                            const float inv = den > 0.f ? 1.0f / den : 0.f;
-                            float *o = p.out + ((int64_t)r * p.Hq + h) * D;
+                            for (int e = 0; e < 2; ++e) {
+                                const int hl = nt * 8 + 2 * t + e;
+                                if (hl >= G) continue;
+                                const int h = g * G + hl;
+                                const float m2 = __ldcg(base + (size_t)p.Hq * D + h);
+                                const float l2 = __ldcg(base + (size_t)p.Hq * (D + 1) + h);
+                                float x[D / 16][2];
 #pragma unroll
-                            for (int nd = 0; nd < D / 8; ++nd)
-                                *reinterpret_cast<float2 *>(o + nd * 8 + 2 * t) = make_float2(
-                                    __fmul_rn(__fadd_rn(__fmul_rn(oacc[nd][2 * i], a), __fmul_rn(x[nd].x, b)), inv),
-                                    __fmul_rn(__fadd_rn(__fmul_rn(oacc[nd][2 * i + 1], a), __fmul_rn(x[nd].y, b)), inv));
-                        }
+                                for (int mt = 0; mt < D / 16; ++mt) {
+                                    x[mt][0] = __ldcg(base + (size_t)h * D + mt * 16 + gid);
+                                    x[mt][1] = __ldcg(base + (size_t)h * D + mt * 16 + 8 + gid);
+                                }
+                                const float mn = fmaxf(m_run[nt][e], m2);
+                                const float a = exp2_or_zero(m_run[nt][e], mn), b = exp2_or_zero(m2, mn);
+                                const float den = __fadd_rn(__fmul_rn(l_run[nt][e], a), __fmul_rn(l2, b));
+                                const float inv = den > 0.f ? 1.0f / den : 0.f;
+                                float *o = p.out + ((int64_t)r * p.Hq + h) * D + gid;
+#pragma unroll
+                                for (int mt = 0; mt < D / 16; ++mt) {
+                                    o[mt * 16] = __fmul_rn(
+                                        __fadd_rn(__fmul_rn(oacc[nt][mt][e], a), __fmul_rn(x[mt][0], b)), inv);
+                                    o[mt * 16 + 8] = __fmul_rn(
+                                        __fadd_rn(__fmul_rn(oacc[nt][mt][2 + e], a), __fmul_rn(x[mt][1], b)), inv);
+                                }
+                            }
                     }
                 } else if (uend == u1 && (size_t)np * slot_floats * 4 <= (size_t)kStages * C::STAGE_BYTES) {
                     // This CTA has no unit left, so the ring is empty: pull all partials of the region into it
