@@ -60,6 +60,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining;
 
+    // the gather kernel that follows may start its text rows now; it waits before it reads the lists
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int r = blockIdx.x;
     const int k = budgets[r];
     int32_t *out = kept + (offsets[r] - (int64_t)r * (n_text + slack));
@@ -168,55 +170,85 @@ struct GatherParams {
 constexpr int kGatherThreads = 256;
 constexpr int kGatherRowsPerWarp = 4;
 
+// Copies the rows of the ragged cache: for region r first the kept visual rows in ascending token order, then
+// the text rows (Algorithm 1's C^l = Concat(K_v[kept], K_t)).  A warp moves four rows at a time.
+// The text rows need no selection result - their place follows from the budgets alone - so they are copied
+// before the kernel waits for its predecessor in the stream (the selection kernel, which releases its
+// dependents at once): that part of the traffic runs beside the selection, which occupies one CTA per region
+// and is bound by latency, not by bandwidth.
 __global__ void __launch_bounds__(kGatherThreads) gather_kernel(GatherParams p) {
     const int lane = threadIdx.x & 31;
-    const int64_t warp_global = ((int64_t)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
+    const int64_t warp0 = ((int64_t)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
+    const int64_t row_step = (int64_t)gridDim.x * (kGatherThreads / 32) * kGatherRowsPerWarp;
     const int n_regions = p.L * p.B;
-    const int64_t total = p.offsets[n_regions];
     const int vec_per_head = p.d / 8;             // 16-byte vectors per head slice
     const int vec_per_row = p.Hkv * vec_per_head;
 
-    int64_t src_off[kGatherRowsPerWarp];
-    int64_t dst_row[kGatherRowsPerWarp];
+    auto copy_rows = [&](const int64_t (&src_off)[kGatherRowsPerWarp], const int64_t (&dst_row)[kGatherRowsPerWarp]) {
+        for (int v0 = lane; v0 < vec_per_row; v0 += 32) {
+            const int g = v0 / vec_per_head, c = v0 % vec_per_head;
+            uint4 kk[kGatherRowsPerWarp], vv[kGatherRowsPerWarp];
 #pragma unroll
-    for (int i = 0; i < kGatherRowsPerWarp; ++i) {
-        const int64_t row = warp_global * kGatherRowsPerWarp + i;
-        dst_row[i] = -1;
-        src_off[i] = 0;
-        if (row >= total) continue;
-        // region r with offsets[r] <= row < offsets[r+1]
-        int lo = 0, hi = n_regions - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (p.offsets[mid] <= row) lo = mid; else hi = mid - 1;
+            for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+                if (dst_row[i] < 0) continue;
+                const int64_t so = src_off[i] + (int64_t)g * p.s_head + c * 8;
+                kk[i] = __ldg(reinterpret_cast<const uint4 *>(p.k + so));
+                vv[i] = __ldg(reinterpret_cast<const uint4 *>(p.v + so));
+            }
+#pragma unroll
+            for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+                if (dst_row[i] < 0) continue;
+                const int64_t dof = (dst_row[i] * p.Hkv + g) * p.d + c * 8;
+                *reinterpret_cast<uint4 *>(p.k_out + dof) = kk[i];
+                *reinterpret_cast<uint4 *>(p.v_out + dof) = vv[i];
+            }
         }
-        const int r = lo;
-        const int64_t base = p.offsets[r];
-        const int j = (int)(row - base);
-        if (j >= p.lens[r]) continue;  // slack row
-        const int n = p.budgets[r];
-        const int l = r / p.B, b = r % p.B;
-        const int tok = j < n ? p.kept[base - (int64_t)r * (p.Nt + p.slack) + j] : p.Nv + (j - n);
-        src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)tok * p.s_token;
-        dst_row[i] = row;
+    };
+
+    // ---- text rows: row j of region r goes to offsets[r] + budgets[r] + j ----
+    const int n_text_rows = n_regions * p.Nt;   // below 2^31: the cache has fewer rows than that
+    for (int64_t first = warp0 * kGatherRowsPerWarp; first < n_text_rows; first += row_step) {
+        int64_t src_off[kGatherRowsPerWarp], dst_row[kGatherRowsPerWarp];
+#pragma unroll
+        for (int i = 0; i < kGatherRowsPerWarp; ++i) {
+            const int idx = (int)first + i;
+            dst_row[i] = -1;
+            src_off[i] = 0;
+            if (idx >= n_text_rows) continue;
+            const int r = idx / p.Nt, j = idx - r * p.Nt;
+            const int l = r / p.B, b = r - l * p.B;
+            src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)(p.Nv + j) * p.s_token;
+            dst_row[i] = p.offsets[r] + p.budgets[r] + j;
+        }
+        copy_rows(src_off, dst_row);
     }
-    for (int v0 = lane; v0 < vec_per_row; v0 += 32) {
-        const int g = v0 / vec_per_head, c = v0 % vec_per_head;
-        uint4 kk[kGatherRowsPerWarp], vv[kGatherRowsPerWarp];
+
+    // ---- kept visual rows, once the selection has written its lists ----
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int64_t per = p.Nt + p.slack;   // offsets[r] - r * per = kept rows of the regions before r
+    const int64_t n_kept = p.offsets[n_regions] - (int64_t)n_regions * per;
+    for (int64_t first = warp0 * kGatherRowsPerWarp; first < n_kept; first += row_step) {
+        int64_t src_off[kGatherRowsPerWarp], dst_row[kGatherRowsPerWarp];
 #pragma unroll
         for (int i = 0; i < kGatherRowsPerWarp; ++i) {
-            if (dst_row[i] < 0) continue;
-            const int64_t so = src_off[i] + (int64_t)g * p.s_head + c * 8;
-            kk[i] = __ldg(reinterpret_cast<const uint4 *>(p.k + so));
-            vv[i] = __ldg(reinterpret_cast<const uint4 *>(p.v + so));
+            const int64_t idx = first + i;
+            dst_row[i] = -1;
+            src_off[i] = 0;
+            if (idx >= n_kept) continue;
+            // largest r with (kept rows before r) <= idx: regions without kept rows are passed over
+            int lo = 0, hi = n_regions - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (p.offsets[mid] - (int64_t)mid * per <= idx) lo = mid; else hi = mid - 1;
+            }
+            const int r = lo;
+            const int64_t base = p.offsets[r];
+            const int j = (int)(idx - (base - (int64_t)r * per));
+            const int l = r / p.B, b = r - l * p.B;
+            src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)p.kept[idx] * p.s_token;
+            dst_row[i] = base + j;
         }
-#pragma unroll
-        for (int i = 0; i < kGatherRowsPerWarp; ++i) {
-            if (dst_row[i] < 0) continue;
-            const int64_t dof = (dst_row[i] * p.Hkv + g) * p.d + c * 8;
-            *reinterpret_cast<uint4 *>(p.k_out + dof) = kk[i];
-            *reinterpret_cast<uint4 *>(p.v_out + dof) = vv[i];
-        }
+        copy_rows(src_off, dst_row);
     }
 }
 
@@ -262,8 +294,26 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     p.L = s->n_layers; p.B = s->batch; p.Hkv = s->n_kv_heads; p.d = s->head_dim;
     p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack;
     const int64_t rows_per_block = (kGatherThreads / 32) * kGatherRowsPerWarp;
-    const int64_t blocks = (p.rows_cap + rows_per_block - 1) / rows_per_block;
-    gather_kernel<<<(unsigned)blocks, kGatherThreads, 0, st>>>(p);
+    const int64_t text_rows = (int64_t)LB * s->n_text;
+    const int64_t kept_rows = p.rows_cap - (int64_t)LB * (s->n_text + s->slack);
+    const int64_t most = text_rows > kept_rows ? text_rows : kept_rows;
+    int dev = 0, sms = 0;
+    AIRCACHE_CUDA_TRY(cudaGetDevice(&dev));
+    AIRCACHE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int64_t blocks = (most + rows_per_block - 1) / rows_per_block;
+    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;   // what is resident at once; the rest is a stride loop
+    if (blocks < 1) blocks = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(kGatherThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    AIRCACHE_CUDA_TRY(cudaLaunchKernelEx(&cfg, gather_kernel, p));
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }
