@@ -176,7 +176,7 @@ constexpr int kGatherRowsPerWarp = 4;
 // before the kernel waits for its predecessor in the stream (the selection kernel, which releases its
 // dependents at once): that part of the traffic runs beside the selection, which occupies one CTA per region
 // and is bound by latency, not by bandwidth.
-__global__ void __launch_bounds__(kGatherThreads) gather_kernel(GatherParams p) {
+__global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams p) {
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
     const int64_t row_step = (int64_t)gridDim.x * (kGatherThreads / 32) * kGatherRowsPerWarp;
@@ -300,8 +300,13 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     int dev = 0, sms = 0;
     AIRCACHE_CUDA_TRY(cudaGetDevice(&dev));
     AIRCACHE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // No more blocks than are resident at once, the rest is a stride loop: a block that only becomes resident
+    // after others have reached their dependency wait would copy its text rows after the selection, not beside it.
+    int per_sm = 0;
+    AIRCACHE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gather_kernel, kGatherThreads, 0));
+    if (per_sm < 1) per_sm = 1;
     int64_t blocks = (most + rows_per_block - 1) / rows_per_block;
-    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;   // what is resident at once; the rest is a stride loop
+    if (blocks > (int64_t)sms * per_sm) blocks = (int64_t)sms * per_sm;
     if (blocks < 1) blocks = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
