@@ -272,7 +272,10 @@ int aircache_selftest_wait_timeout(void *workspace, int64_t workspace_bytes, voi
  * The whole path with HOST inputs and outputs: uploads the full cache and the
  * queries, runs score -> budget -> compact -> n_steps x decode_attn on the
  * stream, downloads the results and synchronises.  Every device buffer is still
- * the caller's (no allocation inside).
+ * the caller's (no device memory is allocated inside).  The outputs of the
+ * decode rounds are copied back in groups of 16 rounds on a second stream that
+ * the call creates and destroys, so that the download overlaps the later rounds;
+ * on return every copy has completed.
  *   h_full       HOST view of the full cache (strides as in aircache_full_t)
  *   full_elems   elements (bf16) spanned by h_full->k and by h_full->v
  *   d_full_k/v   DEVICE buffers of full_elems bf16 each

@@ -327,15 +327,37 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     if ((rc = aircache_compact(shape, &d_full, d_scores, d_budgets, ratio, d_cache, nullptr, workspace,
                                workspace_bytes, st)))
         return rc;
+    // The results go back to the host while later rounds still run: a second stream copies every
+    // kCopyEvery rounds' outputs as soon as the round that wrote the last of them has finished.
+    struct CopySide {
+        cudaStream_t stream = nullptr;
+        cudaEvent_t event = nullptr;
+        ~CopySide() {
+            if (event) cudaEventDestroy(event);
+            if (stream) cudaStreamDestroy(stream);
+        }
+    } side;
+    constexpr int32_t kCopyEvery = 16;
+    if (n_steps > 0) {
+        AIRCACHE_CUDA_TRY(cudaStreamCreateWithFlags(&side.stream, cudaStreamNonBlocking));
+        AIRCACHE_CUDA_TRY(cudaEventCreateWithFlags(&side.event, cudaEventDisableTiming));
+    }
     for (int32_t i = 0; i < n_steps; ++i) {
         const char *q = (const char *)d_q_steps + (int64_t)i * q_elems * 2;
         if ((rc = aircache_decode_attn(shape, d_cache, q, d_out + (int64_t)i * q_elems, workspace,
                                        workspace_bytes, st)))
             return rc;
+        if ((i + 1) % kCopyEvery == 0 || i + 1 == n_steps) {
+            const int32_t first = i / kCopyEvery * kCopyEvery;
+            AIRCACHE_CUDA_TRY(cudaEventRecord(side.event, st));
+            AIRCACHE_CUDA_TRY(cudaStreamWaitEvent(side.stream, side.event, 0));
+            AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_out + (int64_t)first * q_elems, d_out + (int64_t)first * q_elems,
+                                              (int64_t)(i + 1 - first) * q_elems * 4, cudaMemcpyDeviceToHost,
+                                              side.stream));
+        }
     }
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_budgets, d_budgets, LB * 4, cudaMemcpyDeviceToHost, st));
-    if (n_steps > 0)
-        AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_out, d_out, (int64_t)n_steps * q_elems * 4, cudaMemcpyDeviceToHost, st));
+    if (n_steps > 0) AIRCACHE_CUDA_TRY(cudaStreamSynchronize(side.stream));
     AIRCACHE_CUDA_TRY(cudaStreamSynchronize(st));
     return AIRCACHE_OK;
 }
