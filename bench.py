@@ -427,8 +427,9 @@ def describe(wl):
 
 
 def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
-    """Same metric through aircache_pipeline_host: every step uploads the full cache and the queries from
-    pinned host memory, runs the whole path and downloads the attention outputs and the budgets."""
+    """Same metric through aircache_pipeline_host: every step uploads the full K cache and the queries from
+    pinned host memory, reads the surviving V rows from pinned host memory in place, runs the whole path and
+    downloads the attention outputs and the budgets."""
     stream = torch.cuda.current_stream(dev)
     k_tm = s.k_full.permute(0, 1, 3, 2, 4)      # back to the token-major storage order
     v_tm = s.v_full.permute(0, 1, 3, 2, 4)
@@ -451,10 +452,14 @@ def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
     for _ in range(steps):
         once()      # synchronises internally after the device-to-host copies
     dt = (time.perf_counter() - t0) / steps
-    h2d = 2 * h_k.numel() * 2 + h_qw.numel() * 2 + h_q.numel() * 2
+    # K whole; of V (page-locked, read in place by the gather kernel) only the rows of the compressed cache
+    v_in_place = ac.aircache_host_range_is_mapped(h_v)
+    v_bytes = int(s.lens.sum().item()) * wl.n_kv_heads * wl.head_dim * 2 if v_in_place else h_v.numel() * 2
+    h2d = h_k.numel() * 2 + v_bytes + h_qw.numel() * 2 + h_q.numel() * 2
     d2h = h_out.numel() * 4 + h_bud.numel() * 4
     return {"value": n_dec * wl.batch / dt, "unit": UNIT, "ms_per_step": dt * 1e3, "requests_per_step": 1,
-            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "aircache_pipeline_host"}
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "aircache_pipeline_host",
+            "v_read_in_place": bool(v_in_place)}
 
 
 # --------------------------------------------------------------------------------------------------

@@ -269,10 +269,22 @@ int aircache_check_status(void *workspace, int64_t workspace_bytes, void *cuda_s
 int aircache_selftest_wait_timeout(void *workspace, int64_t workspace_bytes, void *cuda_stream);
 
 /*
+ * 1 if the whole host range [host_ptr, host_ptr + bytes) is page-locked memory
+ * that kernels on the current device can read in place, else 0 (pageable
+ * memory, a null pointer, an empty range).  Host-side query, launches nothing.
+ */
+int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes);
+
+/*
  * The whole path with HOST inputs and outputs: uploads the full cache and the
  * queries, runs score -> budget -> compact -> n_steps x decode_attn on the
  * stream, downloads the results and synchronises.  Every device buffer is still
- * the caller's (no device memory is allocated inside).  The outputs of the
+ * the caller's (no device memory is allocated inside).  K is uploaded whole
+ * (the scoring passes read all of it, twice).  V is only ever read where a row
+ * survives: if h_full->v is page-locked host memory that the GPU can address
+ * (cudaHostAlloc / cudaHostRegister; aircache_host_range_is_mapped() tells),
+ * compaction reads the kept and the text rows of V from it in place and
+ * d_full_v stays untouched; otherwise V is uploaded whole like K.  The outputs of the
  * decode rounds are copied back in groups of 16 rounds on a second stream that
  * the call creates and destroys, so that the download overlaps the later rounds;
  * on return every copy has completed.

@@ -75,6 +75,7 @@ _SIGNATURES = {
     "aircache_reset_status": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_check_status": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_selftest_wait_timeout": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
+    "aircache_host_range_is_mapped": (C.c_int, [C.c_void_p, C.c_int64]),
     "aircache_pipeline_host": (C.c_int, [C.POINTER(Shape), C.POINTER(Full), C.c_int64, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float,
                                          C.c_double, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(Ragged),
@@ -242,6 +243,11 @@ def aircache_selftest_wait_timeout(workspace, stream=None, check=True) -> int:
     if check:
         _check("aircache_selftest_wait_timeout", rc)
     return rc
+
+
+def aircache_host_range_is_mapped(host_tensor) -> bool:
+    """True if kernels can read the tensor's host memory in place (page-locked and mapped)."""
+    return bool(lib().aircache_host_range_is_mapped(_ptr(host_tensor), _nbytes(host_tensor)))
 
 
 def aircache_pipeline_host(sh, h_full, full_elems, d_full_k, d_full_v, h_q_window, d_q_window, h_q_steps, d_q_steps,

@@ -286,6 +286,24 @@ int aircache_selftest_wait_timeout(void *workspace, int64_t workspace_bytes, voi
     return launch_selftest_timeout(workspace, (cudaStream_t)cuda_stream);
 }
 
+// Device address of a host range if all of it is page-locked memory the GPU can read in place, else null.
+static void *mapped_host_range(const void *p, int64_t bytes) {
+    if (!p || bytes < 1) return nullptr;
+    void *first = nullptr, *last = nullptr;
+    const char *c = static_cast<const char *>(p);
+    if (cudaHostGetDevicePointer(&first, const_cast<char *>(c), 0) != cudaSuccess ||
+        cudaHostGetDevicePointer(&last, const_cast<char *>(c + bytes - 1), 0) != cudaSuccess) {
+        cudaGetLastError();   // pageable memory: not an error of the caller's, and not a sticky one
+        return nullptr;
+    }
+    if (!first || static_cast<char *>(last) - static_cast<char *>(first) != bytes - 1) return nullptr;
+    return first;
+}
+
+int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes) {
+    return mapped_host_range(host_ptr, bytes) ? 1 : 0;
+}
+
 int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t *h_full, int64_t full_elems,
                            void *d_full_k, void *d_full_v, const void *h_q_window, void *d_q_window,
                            const void *h_q_steps, void *d_q_steps, int32_t n_steps, float alpha, double ratio,
@@ -305,6 +323,11 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     aircache_full_t d_full = *h_full;
     d_full.k = d_full_k;
     d_full.v = d_full_v;
+    // K is read twice in full by the scoring passes, so it is uploaded.  V is read once, and only the rows that
+    // survive (kept visual rows and text rows): when the host buffer is page-locked and mapped, the gather
+    // kernel reads those rows from it in place and the upload of the other rows never happens.
+    void *v_in_place = mapped_host_range(h_full->v, full_elems * 2);
+    if (v_in_place) d_full.v = v_in_place;
     // validate everything the stages will check before the first copy is enqueued
     if ((rc = check_full(shape, &d_full))) return rc;
     if ((rc = check_ragged(shape, d_cache, true))) return rc;
@@ -314,7 +337,8 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
         return AIRCACHE_ERR_INVALID_ARG;
 
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_k, h_full->k, full_elems * 2, cudaMemcpyHostToDevice, st));
-    AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_v, h_full->v, full_elems * 2, cudaMemcpyHostToDevice, st));
+    if (!v_in_place)
+        AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_v, h_full->v, full_elems * 2, cudaMemcpyHostToDevice, st));
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_q_window, h_q_window, qw_bytes, cudaMemcpyHostToDevice, st));
     if (n_steps > 0)
         AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_q_steps, h_q_steps, (int64_t)n_steps * q_elems * 2,

@@ -520,7 +520,11 @@ def test_bounded_wait_ends_in_an_error_code_not_a_hang():
     assert gp.status() == 0 and torch.isfinite(gp.out).all()
 
 
-def test_pipeline_host_matches_staged_calls(oracle):
+@pytest.mark.parametrize("pinned_v", [True, False])
+def test_pipeline_host_matches_staged_calls(oracle, pinned_v):
+    """Host inputs in, host outputs out, equal to the staged calls bit for bit - with V in page-locked memory
+    (compaction reads the surviving rows from it in place; the device buffer for V is poisoned and stays so) and
+    with V in pageable memory (uploaded whole)."""
     import paper_2503_23956_b200 as ac
     wl = CASES["c1"]
     ref = oracle_path(oracle, wl)
@@ -533,9 +537,12 @@ def test_pipeline_host_matches_staged_calls(oracle):
         gp.decode(q_steps[s].to(DEV))
         staged.append(gp.out.cpu().numpy().copy())
     gp2 = GpuPath(wl, ratio=ref["ratio"], device=DEV)
-    h_k, h_v = ref["k"].contiguous().pin_memory(), ref["v"].contiguous().pin_memory()
+    h_k = ref["k"].contiguous().pin_memory()
+    h_v = ref["v"].contiguous().pin_memory() if pinned_v else ref["v"].contiguous().clone()
+    assert ac.aircache_host_range_is_mapped(h_v) == pinned_v
     h_full = ac.full_view(logical(h_k), logical(h_v))
-    d_k, d_v = torch.empty_like(h_k, device=DEV), torch.empty_like(h_v, device=DEV)
+    d_k = torch.empty_like(h_k, device=DEV)
+    d_v = torch.full(h_v.shape, float("nan"), dtype=h_v.dtype, device=DEV)
     h_qw = ref["qw"].contiguous().pin_memory()
     d_qw = torch.empty_like(h_qw, device=DEV)
     h_q = q_steps.pin_memory()
@@ -548,6 +555,7 @@ def test_pipeline_host_matches_staged_calls(oracle):
     assert np.array_equal(h_bud.numpy(), ref["budgets"])
     for s in range(n_steps):
         assert np.array_equal(h_out[s].numpy(), staged[s])
+    assert bool(torch.isnan(d_v.float()).all()) == pinned_v   # V uploaded only when it could not be read in place
 
 
 # --------------------------------------------------------------------------------------------------
