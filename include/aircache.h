@@ -91,12 +91,23 @@ typedef struct {
  * Concat(K_v[kept], K_t) in ascending token order and the rest is slack.
  * aircache_budget writes offsets and lens, aircache_compact writes k and v.
  * k and v must be 128-byte aligned.
+ *
+ * Several caches may share one pair of buffers, packed back to back (requests
+ * whose sequences differ in N_v and N_t, hence in shape, compressed by separate
+ * calls): each call gets the same k, v and total_rows, first_row = the rows
+ * taken by the caches before it (the sum of their aircache_total_rows(), known
+ * on the host), and offsets / lens pointing at its own stretch of two shared
+ * arrays - stretch s starts where stretch s-1 holds its last offset, which is
+ * the same number.  offsets are rows of the shared buffers, so one
+ * aircache_decode_attn call (n_layers = number of all regions, batch = 1) then
+ * attends over all of them.
  */
 typedef struct {
     void *k, *v;
     int64_t *offsets;    /* [L*B + 1] rows */
     int32_t *lens;       /* [L*B]     rows in use */
-    int64_t total_rows;  /* capacity of k and v in rows, >= aircache_total_rows() */
+    int64_t total_rows;  /* capacity of k and v in rows, >= first_row + aircache_total_rows() */
+    int64_t first_row;   /* rows of k and v in front of this cache's first region; 0 for a cache of its own */
 } aircache_ragged_t;
 
 int aircache_version(void);

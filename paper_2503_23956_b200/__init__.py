@@ -46,7 +46,7 @@ class Full(C.Structure):
 
 class Ragged(C.Structure):
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("offsets", C.c_void_p), ("lens", C.c_void_p),
-                ("total_rows", C.c_int64)]
+                ("total_rows", C.c_int64), ("first_row", C.c_int64)]
 
 
 _lib = None
@@ -141,8 +141,9 @@ def full_view(k: torch.Tensor, v: torch.Tensor) -> Full:
     return Full(k.data_ptr(), v.data_ptr(), sl, sb, sh, st)
 
 
-def ragged_view(k, v, offsets, lens, total_rows: int) -> Ragged:
-    return Ragged(_ptr(k), _ptr(v), _ptr(offsets), _ptr(lens), total_rows)
+def ragged_view(k, v, offsets, lens, total_rows: int, first_row: int = 0) -> Ragged:
+    """`offsets` / `lens` may be tensors or raw addresses (a stretch of shared arrays, see aircache_ragged_t)."""
+    return Ragged(_ptr(k), _ptr(v), _ptr(offsets), _ptr(lens), total_rows, first_row)
 
 
 # ------------------------------------------------------------------------------------------------

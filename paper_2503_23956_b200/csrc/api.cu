@@ -88,10 +88,12 @@ static int check_ws(const aircache_shape_t *s, void *ws, int64_t bytes) {
 static int check_ragged(const aircache_shape_t *s, const aircache_ragged_t *c, bool need_kv) {
     if (!c || !c->offsets || !c->lens) return AIRCACHE_ERR_INVALID_ARG;
     if (((uintptr_t)c->offsets & 7) || ((uintptr_t)c->lens & 3)) return AIRCACHE_ERR_ALIGNMENT;
+    if (c->first_row < 0) return AIRCACHE_ERR_INVALID_ARG;
     if (need_kv) {
         if (!c->k || !c->v) return AIRCACHE_ERR_INVALID_ARG;
         if (((uintptr_t)c->k & 127) || ((uintptr_t)c->v & 127)) return AIRCACHE_ERR_ALIGNMENT;
         if (c->total_rows < 1 || c->total_rows >= ((int64_t)1 << 31)) return AIRCACHE_ERR_CAPACITY;
+        if (c->first_row >= c->total_rows) return AIRCACHE_ERR_CAPACITY;
     }
     (void)s;
     return AIRCACHE_OK;
@@ -208,7 +210,7 @@ int aircache_compact(const aircache_shape_t *shape, const aircache_full_t *full,
     if (((uintptr_t)scores & 3) || ((uintptr_t)budgets & 3) || ((uintptr_t)kept_idx & 3))
         return AIRCACHE_ERR_ALIGNMENT;
     if ((rc = check_ragged(shape, out, true))) return rc;
-    if (out->total_rows < aircache_total_rows(shape, ratio)) return AIRCACHE_ERR_CAPACITY;
+    if (out->total_rows < out->first_row + aircache_total_rows(shape, ratio)) return AIRCACHE_ERR_CAPACITY;
     if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
     return launch_compact(shape, full, scores, budgets, ratio, out, kept_idx, workspace,
                           (cudaStream_t)cuda_stream);
@@ -331,7 +333,7 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     // validate everything the stages will check before the first copy is enqueued
     if ((rc = check_full(shape, &d_full))) return rc;
     if ((rc = check_ragged(shape, d_cache, true))) return rc;
-    if (d_cache->total_rows < aircache_total_rows(shape, ratio)) return AIRCACHE_ERR_CAPACITY;
+    if (d_cache->total_rows < d_cache->first_row + aircache_total_rows(shape, ratio)) return AIRCACHE_ERR_CAPACITY;
     if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
     if (!(alpha >= 0.0f && alpha <= 1.0f) || !(ratio >= 0.0 && ratio <= 1.0) || mode < 0 || mode > 3)
         return AIRCACHE_ERR_INVALID_ARG;

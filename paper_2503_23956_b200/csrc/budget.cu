@@ -28,6 +28,7 @@ struct BudgetParams {
     uint32_t *ticket;        // zero between calls
     int L, B, Nv, Nt, slack, mode;
     long long total_kept;    // T per sequence
+    long long first_row;     // rows of the shared buffers in front of this cache's first region
 };
 
 __device__ __forceinline__ double block_sum(double v, double *s_part) {
@@ -248,14 +249,14 @@ __global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
         if (lane < kThreads / 32) s_warp[lane] = vv;
     }
     __syncthreads();
-    long long run = incl - local + (warp > 0 ? s_warp[warp - 1] : 0);
+    long long run = p.first_row + incl - local + (warp > 0 ? s_warp[warp - 1] : 0);
     for (int i = i0; i < i1; ++i) {
         p.offsets[i] = run;
         p.lens[i] = bud[i] + p.Nt;
         p.budgets[i] = bud[i];
         run += bud[i] + p.Nt + p.slack;
     }
-    if (tid == kThreads - 1) p.offsets[LB] = s_warp[kThreads / 32 - 1];
+    if (tid == kThreads - 1) p.offsets[LB] = p.first_row + s_warp[kThreads / 32 - 1];
 }
 
 }  // namespace
@@ -274,6 +275,7 @@ int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, 
     p.ticket = ws_ptr<uint32_t>(ws, w.status) + 2;   // second word pair of the status block
     p.L = s->n_layers; p.B = s->batch; p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack; p.mode = mode;
     p.total_kept = kept_per_sequence(s, ratio);
+    p.first_row = layout->first_row;
     const size_t smem = (size_t)LB * (4 * 8 + 4 + 1) + 16;
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     budget_kernel<<<LB, kThreads, smem, st>>>(p);

@@ -53,7 +53,8 @@ template <bool SMEM_KEYS>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__restrict__ scores,
                                                              const int32_t *__restrict__ budgets,
                                                              const int64_t *__restrict__ offsets, int n_visual,
-                                                             int n_text, int slack, int32_t *__restrict__ kept) {
+                                                             int n_text, int slack, int64_t first_row,
+                                                             int32_t *__restrict__ kept) {
     extern __shared__ uint32_t s_keys[];
     __shared__ int s_hist[256];
     __shared__ int s_warp[kSelThreads / 32];
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int r = blockIdx.x;
     const int k = budgets[r];
-    int32_t *out = kept + (offsets[r] - (int64_t)r * (n_text + slack));
+    int32_t *out = kept + (offsets[r] - first_row - (int64_t)r * (n_text + slack));
     const float *x = scores + (int64_t)r * n_visual;
     if (k <= 0) return;
     if (k >= n_visual) {
@@ -164,6 +165,7 @@ struct GatherParams {
     const int32_t *budgets;
     const int32_t *kept;
     int64_t rows_cap;  // rows covered by the launch
+    int64_t first_row; // rows of the shared buffers in front of this cache's first region
     int L, B, Hkv, d, Nv, Nt, slack;
 };
 
@@ -225,8 +227,8 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
 
     // ---- kept visual rows, once the selection has written its lists ----
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int64_t per = p.Nt + p.slack;   // offsets[r] - r * per = kept rows of the regions before r
-    const int64_t n_kept = p.offsets[n_regions] - (int64_t)n_regions * per;
+    const int64_t per = p.Nt + p.slack;   // offsets[r] - first_row - r * per = kept rows of the regions before r
+    const int64_t n_kept = p.offsets[n_regions] - p.first_row - (int64_t)n_regions * per;
     for (int64_t first = warp0 * kGatherRowsPerWarp; first < n_kept; first += row_step) {
         int64_t src_off[kGatherRowsPerWarp], dst_row[kGatherRowsPerWarp];
 #pragma unroll
@@ -239,11 +241,11 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
             int lo = 0, hi = n_regions - 1;
             while (lo < hi) {
                 const int mid = (lo + hi + 1) >> 1;
-                if (p.offsets[mid] - (int64_t)mid * per <= idx) lo = mid; else hi = mid - 1;
+                if (p.offsets[mid] - p.first_row - (int64_t)mid * per <= idx) lo = mid; else hi = mid - 1;
             }
             const int r = lo;
             const int64_t base = p.offsets[r];
-            const int j = (int)(idx - (base - (int64_t)r * per));
+            const int j = (int)(idx - (base - p.first_row - (int64_t)r * per));
             const int l = r / p.B, b = r - l * p.B;
             src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)p.kept[idx] * p.s_token;
             dst_row[i] = base + j;
@@ -278,10 +280,10 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
         AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                kSelSmemKeys * 4));
         select_kernel<true><<<LB, kSelThreads, smem, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
-                                                           s->slack, kept);
+                                                           s->slack, out->first_row, kept);
     } else {
         select_kernel<false><<<LB, kSelThreads, 0, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
-                                                         s->slack, kept);
+                                                         s->slack, out->first_row, kept);
     }
     AIRCACHE_LAUNCH_CHECK();
 
@@ -290,6 +292,7 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     p.s_layer = f->stride_layer; p.s_batch = f->stride_batch; p.s_head = f->stride_head; p.s_token = f->stride_token;
     p.k_out = (uint16_t *)out->k; p.v_out = (uint16_t *)out->v;
     p.offsets = out->offsets; p.lens = out->lens; p.budgets = budgets; p.kept = kept;
+    p.first_row = out->first_row;
     p.rows_cap = (int64_t)s->batch * (kept_per_sequence(s, ratio) + (int64_t)s->n_layers * (s->n_text + s->slack));
     p.L = s->n_layers; p.B = s->batch; p.Hkv = s->n_kv_heads; p.d = s->head_dim;
     p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack;

@@ -113,6 +113,15 @@ def test_entry_points_reject_bad_arguments_on_the_host():
     assert ac.aircache_compact(sh, full, P, P, 0.5, ac.Ragged(P + 64, P, P, P, 10 ** 6), None, ws, s,
                                check=False) == ac.ERR_ALIGNMENT
     assert ac.aircache_compact(sh, full, None, P, 0.5, rag, None, ws, s, check=False) == ac.ERR_INVALID_ARG
+    # a cache packed behind others in shared buffers: first_row counts against the capacity, and is not negative
+    rows = ac.aircache_total_rows(sh, 0.5)
+    assert ac.aircache_compact(sh, full, P, P, 0.5, ac.Ragged(P, P, P, P, rows + 6, 7), None, ws, s,
+                               check=False) == ac.ERR_CAPACITY
+    assert ac.aircache_compact(sh, full, P, P, 0.5, ac.Ragged(P, P, P, P, rows, -1), None, ws, s,
+                               check=False) == ac.ERR_INVALID_ARG
+    assert ac.aircache_budget(sh, P, 0.5, 0, P, None, None, ac.Ragged(P, P, P, P, rows, -1), ws, s,
+                              check=False) == ac.ERR_INVALID_ARG
+    assert ac.aircache_decode_attn(sh, ac.Ragged(P, P, P, P, 10, 10), P, P, ws, s, check=False) == ac.ERR_CAPACITY
     # decode
     assert ac.aircache_decode_attn(sh, rag, None, P, ws, s, check=False) == ac.ERR_INVALID_ARG
     assert ac.aircache_decode_attn(sh, rag, P, P + 4, ws, s, check=False) == ac.ERR_ALIGNMENT

@@ -9,7 +9,7 @@ import torch
 
 from workloads import CONFIGS, Workload, decode_queries
 
-from harness import GpuPath, gen_inputs, logical, oracle_dims, rel_elem_err, rel_row_err, u16
+from harness import GpuPath, gen_inputs, logical, oracle_dims, rel_elem_err, rel_row_err, shape_of, u16
 
 pytestmark = pytest.mark.gpu
 
@@ -441,6 +441,62 @@ def test_decode_plan_kept_between_calls(oracle, case):
     both(lens2)
     back = both(lens0)
     assert np.array_equal(first, back)
+
+
+@pytest.mark.parametrize("slack", [0, 2])
+def test_sequences_of_different_lengths_share_one_cache(oracle, slack):
+    """Requests whose sequences differ in N_v and N_t are compressed by separate calls into ONE pair of K'/V'
+    buffers (first_row, stretches of shared offsets / lens arrays); a single decode launch then attends over the
+    regions of all of them.  Every request's budgets, kept rows and outputs equal the oracle run on it alone."""
+    import paper_2503_23956_b200 as ac
+    seqs = [small("ragA", L=3, B=1, Nv=1000, Nt=40), small("ragB", L=3, B=1, Nv=515, Nt=64, W=9),
+            small("ragC", L=3, B=1, Nv=300, Nt=20, W=8, ratio=0.33)]
+    refs = [oracle_path(oracle, wl, slack=slack) for wl in seqs]
+    paths = [GpuPath(wl, ratio=ref["ratio"], device=DEV, slack=slack) for wl, ref in zip(seqs, refs)]
+    rows = [ac.aircache_total_rows(gp.sh, ref["ratio"]) for gp, ref in zip(paths, refs)]
+    regions = [wl.n_layers * wl.batch for wl in seqs]
+    total, n_reg = sum(rows), sum(regions)
+    wl0 = seqs[0]
+    k_c = torch.zeros((total, wl0.n_kv_heads, wl0.head_dim), dtype=torch.bfloat16, device=DEV)
+    v_c = torch.zeros_like(k_c)
+    offsets = torch.full((n_reg + 1,), -1, dtype=torch.int64, device=DEV)
+    lens = torch.full((n_reg,), -1, dtype=torch.int32, device=DEV)
+    first_row = first_reg = 0
+    for gp, ref, n_rows, n_r in zip(paths, refs, rows, regions):
+        gp.set_full(logical(ref["k"].to(DEV)), logical(ref["v"].to(DEV)))
+        gp.cache = ac.ragged_view(k_c, v_c, offsets.data_ptr() + 8 * first_reg, lens.data_ptr() + 4 * first_reg, total,
+                                  first_row)
+        run_chain(gp, ref)
+        assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+        cp = ref["compact"]
+        assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+        assert np.array_equal(offsets[first_reg:first_reg + n_r + 1].cpu().numpy(), cp["offsets"] + first_row)
+        assert np.array_equal(lens[first_reg:first_reg + n_r].cpu().numpy(), cp["lens"])
+        kc, vc = u16(k_c), u16(v_c)
+        for r in range(n_r):
+            a, n = int(cp["offsets"][r]), int(cp["lens"][r])
+            assert np.array_equal(kc[first_row + a:first_row + a + n], cp["k"][a:a + n])
+            assert np.array_equal(vc[first_row + a:first_row + a + n], cp["v"][a:a + n])
+        first_row += n_rows
+        first_reg += n_r
+    assert int(offsets[-1].item()) == total
+    # one launch over all regions: a shape with as many "layers" as there are regions, batch 1
+    sh_all = shape_of(wl0, n_layers=n_reg, batch=1, slack=slack)
+    cache_all = ac.ragged_view(k_c, v_c, offsets, lens, total)
+    qs = [decode_queries(wl, 0, "cpu") for wl in seqs]
+    q_all = torch.cat([q.reshape(-1, wl0.n_q_heads, wl0.head_dim) for q in qs]).contiguous().to(DEV)
+    out = torch.full((n_reg, wl0.n_q_heads, wl0.head_dim), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(ac.aircache_workspace_bytes(sh_all), dtype=torch.uint8, device=DEV)
+    ac.aircache_reset_status(ws)
+    ac.aircache_decode_attn(sh_all, cache_all, q_all, out, ws)
+    assert ac.aircache_check_status(ws, check=False) == 0
+    got = out.cpu().numpy()
+    first_reg = 0
+    for wl, ref, q, n_r in zip(seqs, refs, qs, regions):
+        cp = ref["compact"]
+        want = oracle.decode(ref["dims"], cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q), wl.scale)
+        assert rel_row_err(got[first_reg:first_reg + n_r], want) <= TOL
+        first_reg += n_r
 
 
 def _random_workload(seed):
