@@ -16,6 +16,7 @@ layers of a real model.
                   call / average duration of a call inside the timed region
   e2e             the same metric through aircache_pipeline_host: pinned host inputs, host outputs
   cpu_baseline    the CPU oracle timed on this host (rank 0, N = 1 only)
+  allocation_ablation   budget vectors of the four allocation rules (mode flag) and their JS divergence
   hbm_bound_workloads   the decode and compaction rooflines on further workloads (default: config 4, 261 MB
                   per decode launch), measured briefly after the main run at N = 1
 
@@ -38,6 +39,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 METRIC = "decode_tok_s_at_10pct_visual_kv"
@@ -359,6 +361,7 @@ def run_cuda(args):
     if rank == 0 and not args.no_e2e:
         result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 5))
     if rank == 0 and world == 1 and args.extra not in ("", "none"):
+        result["allocation_ablation"] = allocation_ablation(ac, wl, reqs[0])
         result["score_dense_window"] = dense_window_score(wl, reqs[0])
     del reqs
     torch.cuda.empty_cache()
@@ -419,6 +422,36 @@ def dense_window_score(wl, s, reps=10):
     return {"alpha": 0.0, "rows_per_kv_group": rows, "us_per_request": us, "tflops": flops / (us * 1e-6) / 1e12,
             "key_bytes": wl.n_visual * wl.n_kv_heads * wl.head_dim * 2 * wl.n_layers * wl.batch,
             "note": "both passes of Eq. 7 on tcgen05; FLOPs count the unpadded rows, keys are read once per pass"}
+
+
+def allocation_ablation(ac, wl, s):
+    """The allocation variants of the paper's ablation (strength + skewness, strength only, skewness only,
+    uniform) as budget vectors over the layers of sequence 0, from aircache_budget's mode flag on the scores of
+    one resident request, and the Jensen-Shannon divergence (bits) of every variant's distribution of the budget
+    over the layers from the combined rule's."""
+    s.score(s.qw)
+    LB = wl.n_layers * wl.batch
+    budgets = torch.empty_like(s.budgets)
+    layout = ac.ragged_view(None, None, torch.empty(LB + 1, dtype=torch.int64, device=s.dev),
+                            torch.empty(LB, dtype=torch.int32, device=s.dev), 0)
+    names = ["strength_and_skewness", "strength_only", "skewness_only", "uniform"]
+    vec = {}
+    for mode, name in enumerate(names):
+        ac.aircache_budget(s.sh, s.scores, s.ratio, mode, budgets, None, None, layout, s.ws)
+        vec[name] = budgets[:, 0].cpu().numpy().astype(np.float64)
+
+    def js(a, b):
+        pa, pb = a / max(a.sum(), 1.0), b / max(b.sum(), 1.0)
+        m = 0.5 * (pa + pb)
+
+        def kl(x, y):
+            nz = x > 0
+            return float(np.sum(x[nz] * np.log2(x[nz] / y[nz])))
+        return 0.5 * kl(pa, m) + 0.5 * kl(pb, m)
+
+    ref = vec[names[0]]
+    return {"budgets_per_layer_sequence0": {n: [int(x) for x in v] for n, v in vec.items()},
+            "js_divergence_bits_vs_combined": {n: js(vec[n], ref) for n in names[1:]}}
 
 
 def describe(wl):
