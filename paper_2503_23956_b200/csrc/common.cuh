@@ -16,8 +16,9 @@ constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode gr
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int64_t kStatusBytes = 256 + (int64_t)kMaxRegions * 4;  // status word + tickets, at the start of the workspace
-// Head-split decode launches (at least two KV heads per region, so at most kMaxDecodeCtas / 2 regions) keep, per
-// CTA, the plan of their last call: 16 words of outcome and the unit count of every region.
+// Decode launches over few regions plan per warp, in registers (head-split launches: at least two KV heads per
+// region, so at most kMaxDecodeCtas / 2 regions; by-region launches: up to 64 regions), and keep, per CTA, the
+// plan of their last call: 16 words of outcome and the unit count of every region.
 constexpr int kPlanRegionsPerLane = kMaxDecodeCtas / 2 / 32;
 constexpr int kPlanMemoInts = 16 + 32 * kPlanRegionsPerLane;
 constexpr int64_t kPlanMemoBytes = (int64_t)kMaxDecodeCtas * kPlanMemoInts * 4;

@@ -179,6 +179,11 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
 // Returns 0 when the tables have to decide (empty regions, too many regions, no fitting cut), 2 when this CTA
 // has no piece, 1 with plan = {item, rows of the item, first unit, end unit} and the item's table entries
 // stored if `store` is set (units counted from the item's first one).
+// With BALANCED set (the by-region kernels) a cut that does not fit is no reason to give up: the warp then
+// writes the unit prefix and first row of every region into the shared tables itself (every warp writes the
+// same values, none waits for another) and returns 3 with plan = {-1, total units, first unit, end unit} of the
+// balanced schedule, CTA c taking units [c * upc, (c + 1) * upc) of the global list; `force_balanced` makes the
+// rehearsal take that way.  RPL = regions a lane may hold.
 //
 // `memo` (may be null) points at this CTA's kPlanMemoInts words of global memory, zero before their first use.
 // The cut depends on the regions' unit counts alone, and those change only every CH appended tokens, so the CTA
@@ -188,10 +193,10 @@ __device__ __forceinline__ int find_region(const int *P, int n, int u) {
 // in shared memory, hence the plain loads).
 //   words 0..4: n, hs, n_ctas, ch_log2, outcome (1 or 2);  8..13: item, first unit, end unit, units, first CTA of the
 //   item, pieces;  14: region;  16..: unit count of every region
+template <int RPL, bool BALANCED>
 __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64_t *offsets, int n, int hs, int n_ctas,
-                                                int ch_log2, int c, bool store, int32_t *memo, int *s_P, int *s_off,
-                                                int *s_Q, int4 *plan) {
-    constexpr int RPL = kPlanRegionsPerLane;
+                                                int ch_log2, int c, bool store, bool force_balanced, int32_t *memo,
+                                                int *s_P, int *s_off, int *s_Q, int4 *plan) {
     const int lane = threadIdx.x & 31;
     const int nr = n / hs;
     if (n > n_ctas || nr <= 0 || nr > 32 * RPL) return 0;
@@ -283,7 +288,36 @@ __device__ __forceinline__ int plan_few_regions(const int32_t *lens, const int64
     sum1 = __reduce_add_sync(0xffffffffu, sum1);
     sum2 = __reduce_add_sync(0xffffffffu, sum2);
     const int lim = n_ctas / hs;   // the sums count pieces per head
-    if (sum0 > lim && sum1 > lim && sum2 > lim) return 0;
+    if ((sum0 > lim && sum1 > lim && sum2 > lim) || (BALANCED && force_balanced)) {
+        if (!BALANCED) return 0;
+        // balanced schedule: exclusive prefix of the unit counts, written by every lane for its regions
+        int mine_units = 0;
+#pragma unroll
+        for (int j = 0; j < RPL; ++j) mine_units += un[j];
+        int incl_units = mine_units;
+#pragma unroll
+        for (int sh = 1; sh < 32; sh <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl_units, sh);
+            if (lane >= sh) incl_units += o;
+        }
+        if (store) {
+            int before = incl_units - mine_units;
+#pragma unroll
+            for (int j = 0; j < RPL; ++j) {
+                const int reg = lane * rpl + j;
+                if (j < rpl && reg < nr) {
+                    s_P[reg] = before;
+                    s_off[reg] = of[j];
+                    before += un[j];
+                    if (reg == nr - 1) s_P[nr] = before;
+                }
+            }
+        }
+        __syncwarp();
+        const int u_first = min(tot, c * upc);
+        *plan = make_int4(-1, tot, u_first, min(tot, u_first + upc));
+        return 3;
+    }
     int pc[RPL];
     int mine = 0;
 #pragma unroll
@@ -399,22 +433,27 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s_abort = 0;
     }
-    // made-up region lengths (one unit each) and first rows for the rehearsal of the register plan below
-    constexpr int kPlanRegions = 32 * kPlanRegionsPerLane;
+    // made-up region lengths (one unit each), first rows and a kept plan that matches them, for the rehearsal of
+    // the register plan below
+    // (head-split launches have at least two heads per region; with more than 64 regions the by-region kernels
+    // measured no faster through the registers than through the shared tables)
+    constexpr int kPlanRpl = HS ? kPlanRegionsPerLane : 2;
+    constexpr int kPlanRegions = 32 * kPlanRpl;
     int32_t *rehearsal_lens = reinterpret_cast<int32_t *>(s_part);
     int64_t *rehearsal_offsets = reinterpret_cast<int64_t *>(s_part + kPlanRegions);
-    int32_t *rehearsal_memo = reinterpret_cast<int32_t *>(s_part + 3 * kPlanRegions);   // a kept plan that matches them
-    if (HS && tid < kPlanRegions) {
-        rehearsal_lens[tid] = CH;
-        rehearsal_offsets[tid] = 0;
-        rehearsal_memo[16 + tid] = tid < n / hs ? 1 : 0;
-        if (tid < 16) {
+    int32_t *rehearsal_memo = reinterpret_cast<int32_t *>(s_part + 3 * kPlanRegions);
+    static_assert((3 * kPlanRegions + kPlanMemoInts) * 4 <= C::SCRATCH_BYTES, "rehearsal inputs fit the scratch area");
+    for (int i = tid; i < kPlanRegions; i += C::THREADS) {
+        rehearsal_lens[i] = CH;
+        rehearsal_offsets[i] = 0;
+        rehearsal_memo[16 + i] = i < n / hs ? 1 : 0;
+        if (i < 16) {
             // n, hs, n_ctas, log2 CH, outcome 1 | item 0 = units [0, 1) of 1, first CTA 0, one piece, region 0
             const int words[16] = {n, hs, n_ctas, C::CH_LOG2, 1, 0, 0, 0, 0, 0, 1, 1, 0, 1, 0, 0};
             int w = 0;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) if (tid == i) w = words[i];
-            rehearsal_memo[tid] = w;
+            for (int k = 0; k < 16; ++k) if (i == k) w = words[k];
+            rehearsal_memo[i] = w;
         }
     }
     // The barriers are initialised before any warp goes its own way (nothing above read global memory).
@@ -439,35 +478,39 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
     // ---- few regions: every warp plans for itself, in registers; otherwise the tables below decide ----
     bool planned = false;
-    if constexpr (HS) {   // head-split launches are the ones with few items; the by-region kernels keep their registers
+    {
         // The plan runs twice through the same instructions: first on the made-up lengths in shared memory (with a
-        // kept plan that matches them, the usual case), while the kernel may not read global memory yet, then on
-        // the real ones.  A kernel's first pass through a
-        // stretch of code waits for its instructions line by line, which for this serial stretch costs more than
-        // its arithmetic; the rehearsal moves that wait in front of the dependency wait, where the CTA idles.
+        // kept plan that matches them, the usual case of a head-split launch; the by-region kernels rehearse the
+        // balanced schedule), while the kernel may not read global memory yet, then on the real ones.  A kernel's
+        // first pass through a stretch of code waits for its instructions line by line, which for this serial
+        // stretch costs more than its arithmetic; the rehearsal moves that wait in front of the dependency wait,
+        // where the CTA idles.
         int4 plan;
         int rc = 0;
+        const bool few = n <= n_ctas && n / hs <= kPlanRegions;   // else only the wait remains of the loop below
 #pragma unroll 1
-        for (int pass = 0; pass < 2; ++pass) {
+        for (int pass = few ? 0 : 1; pass < 2; ++pass) {
             if (pass) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
                 DECODE_TRACE(16);
+                if (!few) break;
             }
-            rc = plan_few_regions(pass ? p.lens : rehearsal_lens, pass ? p.offsets : rehearsal_offsets, n, hs, n_ctas,
-                                  C::CH_LOG2, (int)blockIdx.x, pass != 0,
-                                  !p.plan_memo ? nullptr
-                                               : (pass ? p.plan_memo + (size_t)blockIdx.x * kPlanMemoInts : rehearsal_memo),
-                                  s_P, s_off, s_Q, &plan);
+            rc = plan_few_regions<kPlanRpl, !HS>(
+                pass ? p.lens : rehearsal_lens, pass ? p.offsets : rehearsal_offsets, n, hs, n_ctas, C::CH_LOG2,
+                (int)blockIdx.x, pass != 0, pass == 0,
+                !p.plan_memo ? nullptr
+                             : (pass ? p.plan_memo + (size_t)blockIdx.x * kPlanMemoInts : (HS ? rehearsal_memo : nullptr)),
+                s_P, s_off, s_Q, &plan);
         }
         if (rc == 2) { finish(true); return; }
         if (rc == 1) {
             planned = aligned = true;
             r_own = plan.x; len_own = plan.y; u0 = plan.z; u1 = plan.w;
+        } else if (rc == 3) {
+            planned = true;
+            total = plan.y; u0 = plan.z; u1 = plan.w;
+            upc = max(1, small_div(total + n_ctas - 1, n_ctas));
         }
-    }
-    else {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        DECODE_TRACE(16);
     }
     DECODE_TRACE(12);
     if (!planned) {
