@@ -456,6 +456,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             rehearsal_memo[i] = w;
         }
     }
+    // Ask for the lines the plan will read first (lengths, first rows, this CTA's kept plan) to be brought into
+    // L2 meanwhile: a prefetch consumes no value, so it may precede the dependency wait, and the loads after the
+    // wait then find L2 instead of HBM.
+    if (wid == NCW) {
+        const int n_reg = n / hs;
+        const char *lines[3] = {reinterpret_cast<const char *>(p.lens), reinterpret_cast<const char *>(p.offsets),
+                                reinterpret_cast<const char *>(p.plan_memo ? p.plan_memo + (size_t)blockIdx.x * kPlanMemoInts
+                                                                           : nullptr)};
+        const int bytes[3] = {n_reg * 4, n_reg * 8, HS || n_reg <= 64 ? (16 + n_reg) * 4 : 0};
+#pragma unroll
+        for (int a = 0; a < 3; ++a)
+            if (lines[a] != nullptr && lane * 128 < bytes[a] && lane < 16)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(lines[a] + lane * 128) : "memory");
+    }
     // The barriers are initialised before any warp goes its own way (nothing above read global memory).
     __syncthreads();
 
