@@ -2,26 +2,30 @@
 // decoding), all layers and sequences in one persistent launch.
 //
 // Work decomposition.  A "unit" is CH consecutive rows of one region (all KV heads, K and V).  Region r
-// has ceil(lens[r] / CH) units; every CTA first scans these counts into a prefix P (shared memory), then
-// takes the contiguous unit range [c * upc, (c+1) * upc) of the global unit list, upc = ceil(total / CTAs).
-// The load is therefore balanced to one unit regardless of how ragged the regions are.  When there are
-// few regions and cutting each one into pieces of at most upc units needs no more CTAs than the grid has,
-// the pieces are aligned to regions instead (same longest piece, but one query load and one flush per CTA).  Consecutive units
-// of one region accumulate in registers; a region that lies wholly inside one CTA's range is finished and
-// written by that CTA, otherwise the CTA writes an unnormalised partial (running max, sum, accumulator) and
-// takes a ticket of the region; the CTA that draws the last ticket merges the region's partials in CTA
-// order (split-K with a fixed combination order, whoever arrives last) and puts the ticket back to zero
-// for the next call.  Nobody waits for anybody.
+// has ceil(lens[r] / CH) units; the units of all regions form one list, and CTA c takes the contiguous
+// range [c * upc, (c+1) * upc) of it, upc = ceil(total / CTAs): the load is balanced to one unit however
+// ragged the regions are.  When there are few regions and cutting each one into pieces needs no more CTAs
+// than the grid has, the pieces are aligned to regions instead (one query load and one flush per CTA).
+// When even (region, KV head) pairs do not outnumber the CTAs, the launcher cuts by such pairs
+// ("head-split": the one-KV-head instantiation, the head taken from the item index).  With many regions
+// every CTA builds the unit prefix in shared memory (block-wide scan); with few, every warp derives the
+// handful of numbers it needs in registers (plan_few_regions), rehearsed before the dependency wait and
+// kept in the workspace between calls.  Consecutive units of one region accumulate in registers; a region
+// that lies wholly inside one CTA's range is finished and written by that CTA, otherwise the CTA writes
+// an unnormalised partial (running max, sum, accumulator) and takes a ticket of the region; the CTA that
+// draws the last ticket merges the region's partials (split-K with a result that does not depend on who
+// arrives last) and puts the ticket back to zero for the next call.  Nobody waits for anybody.
 //
 // Inside a CTA.  One producer warp streams units through a ring of shared-memory stages with TMA
 // (cp.async.bulk.tensor, 128-byte swizzle, one box of CH rows x 64 channels per KV head and half of
-// head_dim) and mbarriers.  Consumer warp (g, ks) owns KV head g and the 16-row block ks of every unit:
-//   S = Q_g K^T   mma.m16n8k16: the G query heads of the group are the M rows (padded to 16), keys are N;
-//                 K fragments come from ldmatrix on the swizzled tile
-//   online softmax in the exp2 domain, warp-shuffle row maxima over the quad that shares a row
-//   O += P V      P split into a bf16 head and a bf16 remainder (two MMAs per V fragment: a single bf16
-//                 rounding of P costs up to 2^-9 relative, too close to the 2e-3 bar), V fragments from
-//                 ldmatrix.trans
+// head_dim) and mbarriers.  Consumer warp (g, ks) owns KV head g and the 16-row block ks of every unit;
+// both products are taken transposed, so that the 8 tile columns are the query heads of the KV group:
+//   S^T = K Q_g^T   mma.m16n8k16: the 16 keys are the M rows (K fragments from ldmatrix on the swizzled
+//                   tile), the G query heads the N columns (two column tiles for 9-16 heads)
+//   online softmax in the exp2 domain, column maxima over the eight lanes that share a head pair
+//   O^T += V^T P^T  P split into a bf16 head and a bf16 remainder (two MMAs per V fragment: a single bf16
+//                   rounding of P costs up to 2^-9 relative, too close to the 2e-3 bar), moved into the
+//                   operand layout with movmatrix; V^T fragments from ldmatrix.trans
 // The G-fold reuse of every K/V row across the query heads of a group is what puts this on the tensor
 // pipe: with plain FMAs the kernel would need about 7 flop per byte, more than half of the fp32 peak at
 // full HBM rate.
