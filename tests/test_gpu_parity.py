@@ -33,6 +33,8 @@ CASES = {
     "kv1long": small("kv1long", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=9000, Nt=9, W=4, ratio=0.9),
     # more (region, KV head) pairs than SMs: the by-region decode schedule with several regions per CTA
     "many": small("many", L=10, Hq=28, Hkv=4, d=128, B=4, Nv=300, Nt=20, W=8),
+    # the largest number of regions the library takes (L * B = 1792), each of them tiny
+    "maxreg": small("maxreg", L=28, Hq=8, Hkv=2, d=64, B=64, Nv=40, Nt=4, W=4, ratio=0.25),
 }
 
 
@@ -279,7 +281,7 @@ def run_chain(gp, ref):
     gp.compact()
 
 
-@pytest.mark.parametrize("case", ["c1", "s7b", "s72b", "kv2"])
+@pytest.mark.parametrize("case", ["c1", "s7b", "s72b", "kv2", "maxreg"])
 def test_end_to_end_chain(oracle, case):
     wl = CASES[case]
     ref = oracle_path(oracle, wl)
