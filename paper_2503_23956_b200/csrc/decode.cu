@@ -713,6 +713,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
             }
         }
+        if (p.k_new != nullptr && r_own >= 0) {
+            // Eq. 2 bookkeeping off the critical path: a CTA planned in registers needs lens no more (its row
+            // count sits in registers), so its idle producer draws the ticket now instead of the consumers at
+            // the end; lens is bumped by whoever draws the last ticket, when no CTA will read it again.
+            int last = 0;
+            if (lane == 0) {
+                last = atomicAdd(p.done_ticket, 1) == n_ctas - 1;
+                if (last) *p.done_ticket = 0;
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last)
+                for (int i = lane; i < n / hs; i += 32) p.lens_rw[i] += 1;
+        }
         return;
     }
 
@@ -848,6 +861,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     };
 
     // Writes the region's result (whole region inside this CTA) or an unnormalised partial.
+    uint4 tok = make_uint4(0u, 0u, 0u, 0u);
+    bool tok_ready = false;
+    // 16 bytes of the appended token's row of item r: lanes 0-15 chunk c of K, lanes 16-31 chunk c of V
+    auto load_token = [&](int r) {
+        const int reg = r / hs, head = HS ? r % hs : g;
+        const int64_t src = ((int64_t)reg * p.kv_heads + head) * D;
+        const int c = lane & 15;
+        const uint16_t *from = lane < 16 ? p.k_new : p.v_new;
+        return c < D / 8 ? __ldg(reinterpret_cast<const uint4 *>(from + src) + c) : make_uint4(0u, 0u, 0u, 0u);
+    };
     auto flush = [&](int r, int ustart, int uend) {
         if (p.k_new != nullptr && uend == s_P[r + 1]) {
             // Eq. 2: this CTA holds the item's last unit, so the appended token joins here.  Warp ks = 0 of every
@@ -855,15 +878,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // tile are whatever lies behind it: masked like any row past the end), stores them into the cache
             // and runs the block routine on it.
             if (ks == 0) {
-                const int reg = r / hs, head = HS ? r % hs : g;
+                const int head = HS ? r % hs : g;
                 uint8_t *area = reinterpret_cast<uint8_t *>(s_merge) + g * (4 * 128);
-                const int64_t src = ((int64_t)reg * p.kv_heads + head) * D;
                 const int64_t dst = (((int64_t)s_off[r] + len) * p.kv_heads + head) * D;
                 const int c = lane & 15;
+                const uint4 v = tok_ready ? tok : load_token(r);
+                tok_ready = false;
                 if (c < D / 8) {
-                    const uint16_t *from = lane < 16 ? p.k_new : p.v_new;
                     uint16_t *to = lane < 16 ? p.k_cache : p.v_cache;
-                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(from + src) + c);
                     *reinterpret_cast<uint4 *>(area + (lane < 16 ? 0 : 2 * 128) + (c >> 3) * 128 + (c & 7) * 16) = v;
                     reinterpret_cast<uint4 *>(to + dst)[c] = v;
                 }
@@ -1112,6 +1134,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     int seg_start = u0;
     len = r_own >= 0 ? len_own : p.lens[r / hs];
     load_q(r);
+    // Eq. 2: when this CTA will flush the item's last unit, the appended token's K (lanes 0-15) and V (lanes 16-31)
+    // are requested now, so that the flush does not wait for them
+    if (p.k_new != nullptr && ks == 0 && r_own >= 0 && u1 == s_P[r + 1]) {
+        tok = load_token(r);
+        tok_ready = true;
+    }
     DECODE_TRACE(18);
     int it = 0;
     bool ok = true;
@@ -1140,7 +1168,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     }
     DECODE_TRACE(3 + 3 * n_flush);
     if (ok) flush(r, seg_start, u1);
-    finish(false);
+    if (r_own < 0) finish(false);   // (else the producer warp has drawn the ticket already)
     DECODE_TRACE(5 + 3 * n_flush);
     DECODE_TRACE(15);
     (void)n_flush;
