@@ -386,7 +386,7 @@ def run_cuda(args):
             torch.cuda.empty_cache()
         result["hbm_bound_workloads"] = extra
         # Eq. 2: the same decode rounds with one new token's K/V appended to every region in each round
-        # (the cache grows over the rounds; lens change, so every launch re-derives its schedule)
+        # (the cache grows over the rounds: lens change with every launch)
         d3 = min(n_dec, 64)
         m3, q3 = measure(ac, wl, d3, rotate, 3, 3, not args.no_graph, dev, rank, None, append=True)
         result["decode_with_append"] = {
