@@ -445,6 +445,36 @@ def test_decode_plan_kept_between_calls(oracle, case):
     assert np.array_equal(first, back)
 
 
+def test_one_workspace_serves_different_caches_in_turn(oracle):
+    """The plans a decode launch keeps in the workspace belong to the unit counts it saw: two caches of the same
+    shape but different retention ratios (other lengths, other unit counts) decode alternately through ONE
+    workspace, and every result is the one the cache gets with a workspace of its own."""
+    import paper_2503_23956_b200 as ac
+    wl = CASES["s7b"]
+    refs = [oracle_path(oracle, wl, ratio=0.1), oracle_path(oracle, wl, ratio=0.6)]
+    paths = [make_gpu(wl, ref) for ref in refs]
+    for gp, ref in zip(paths, refs):
+        run_chain(gp, ref)
+    q = decode_queries(wl, 0, "cpu")
+    qd = q.to(DEV)
+    wants = [oracle.decode(ref["dims"], ref["compact"]["k"], ref["compact"]["v"], ref["compact"]["offsets"],
+                           ref["compact"]["lens"], u16(q), wl.scale) for ref in refs]
+    own = []
+    for gp in paths:
+        gp.decode(qd)
+        own.append(gp.out.cpu().numpy().copy())
+    shared_ws = paths[0].ws
+    for turn in range(6):
+        i = turn % 2 if turn < 4 else 1          # A B A B B B: misses, then hits
+        gp = paths[i]
+        gp.out.fill_(float("nan"))
+        ac.aircache_decode_attn(gp.sh, gp.cache, qd, gp.out, shared_ws)
+        assert ac.aircache_check_status(shared_ws, check=False) == 0
+        got = gp.out.cpu().numpy()
+        assert np.array_equal(got, own[i])
+        assert rel_row_err(got, wants[i]) <= TOL
+
+
 @pytest.mark.parametrize("slack", [0, 2])
 def test_sequences_of_different_lengths_share_one_cache(oracle, slack):
     """Requests whose sequences differ in N_v and N_t are compressed by separate calls into ONE pair of K'/V'
