@@ -32,8 +32,10 @@
  *             argument checks run on the host before anything is launched, so a
  *             failing call has enqueued nothing.  No exception crosses the ABI.
  * Threads.    The library keeps no mutable global state apart from a per-thread
- *             copy of the last CUDA error code; calls that share a workspace must
- *             be ordered on one stream.
+ *             copy of the last CUDA error code and the device address of the
+ *             built-in array of aircache_decode_attn_static (looked up once per
+ *             device, under a lock); calls that share a workspace must be ordered
+ *             on one stream.
  * Determinism. Same inputs give the same output bits on every run.
  */
 #ifndef AIRCACHE_H
