@@ -18,7 +18,8 @@ layers of a real model.
   cpu_baseline    the CPU oracle timed on this host (rank 0, N = 1 only)
   allocation_ablation   budget vectors of the four allocation rules (mode flag) and their JS divergence
   hbm_bound_workloads   the decode and compaction rooflines on further workloads (default: config 4, 261 MB
-                  per decode launch), measured briefly after the main run at N = 1
+                  per decode launch, and config 3 at batch 16 and 64, 0.5 and 2 GB per launch), measured briefly
+                  after the main run at N = 1
 
 `python bench.py --impl reference` times the CPU oracle instead (there is no other implementation of the
 paper's method to run).  Under torchrun every rank runs the same workload on its own GPU with its own seeds
@@ -64,7 +65,7 @@ def parse_args():
     ap.add_argument("--decode-steps", type=int, default=0, help="decode rounds per step (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--extra", default="c4", help="comma list of further workloads measured briefly at N = 1 "
+    ap.add_argument("--extra", default="c4,c3:16,c3:64", help="comma list of further workloads measured briefly at N = 1 "
                                                   "(decode and compaction rooflines); \"none\" to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
