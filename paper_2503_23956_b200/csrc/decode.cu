@@ -586,7 +586,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // pieces need no more CTAs than the grid has (two more units on the longest CTA cost less than a
             // second flush and merge).  All items of a region have the same unit count, so the sums run over
             // regions; the three candidates are evaluated together.  Rolled loops: this runs once.
-            const bool few = n <= n_ctas && total > 0;
+            // With more than half as many regions as CTAs an aligned cut would have to leave most regions
+            // whole, which pieces of about total / CTAs units cannot do unless the regions are tiny: the search
+            // is skipped there (it costs over a microsecond on a hundred regions) and the schedule is balanced.
+            const bool few = n <= n_ctas && total > 0 && !(2 * n > n_ctas && upc > 4);
             const int nr = n / hs;
             int sum0 = 0, sum1 = 0, sum2 = 0;
     #pragma unroll 1
