@@ -49,7 +49,7 @@ L2_BYTES = 126 * 2 ** 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from the ncu capture summarised
 # in profiles/; valid only for the kernel source it was taken on (sha1 of csrc/decode.cu, first 12 hex).
-NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "f43881964fa9", "bytes_per_launch": 49492000}
+NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "c37c1ce85fef", "bytes_per_launch": 49489000}
 
 
 def parse_args():
