@@ -372,18 +372,22 @@ def run_cuda(args):
     if rank == 0 and world == 1 and args.extra not in ("", "none"):
         extra = {}
         for spec in args.extra.split(","):
-            w2 = pick_workload(spec, None)
-            r2, _ = default_rotate(ac, w2)
-            d2 = min(w2.steps, 32)
-            m2, q2 = measure(ac, w2, d2, r2, 3, 3, not args.no_graph, dev, rank, None)
-            dec2, comp2 = rooflines(ac, w2, m2, r2, d2)
-            extra[spec] = {"workload": describe(w2), "decode_steps": d2, "resident_requests": r2,
-                           "decode_tok_s": r2 * d2 * w2.batch / (m2["stage_ms"]["decode"] * 1e-3),
-                           "compress_us_per_layer": (m2["stage_ms"]["score"] + m2["stage_ms"]["budget"] +
-                                                     m2["stage_ms"]["compact"]) * 1e3 / (r2 * w2.n_layers),
-                           "stage_us_per_request": {k: v * 1e3 / r2 for k, v in m2["stage_ms"].items()},
-                           "roofline": dec2, "roofline_compact": comp2, "clocks": m2["clocks"]}
-            del q2
+            try:
+                w2 = pick_workload(spec, None)
+                r2, _ = default_rotate(ac, w2)
+                d2 = min(w2.steps, 32)
+                m2, q2 = measure(ac, w2, d2, r2, 3, 3, not args.no_graph, dev, rank, None)
+                dec2, comp2 = rooflines(ac, w2, m2, r2, d2)
+                extra[spec] = {"workload": describe(w2), "decode_steps": d2, "resident_requests": r2,
+                               "decode_tok_s": r2 * d2 * w2.batch / (m2["stage_ms"]["decode"] * 1e-3),
+                               "compress_us_per_layer": (m2["stage_ms"]["score"] + m2["stage_ms"]["budget"] +
+                                                         m2["stage_ms"]["compact"]) * 1e3 / (r2 * w2.n_layers),
+                               "stage_us_per_request": {k: v * 1e3 / r2 for k, v in m2["stage_ms"].items()},
+                               "roofline": dec2, "roofline_compact": comp2, "clocks": m2["clocks"]}
+                del q2
+            except torch.cuda.OutOfMemoryError as e:
+                # a further workload that does not fit this GPU's free memory does not take the main line down
+                extra[spec] = {"skipped": f"out of device memory: {str(e)[:120]}"}
             torch.cuda.empty_cache()
         result["hbm_bound_workloads"] = extra
         # Eq. 2: the same decode rounds with one new token's K/V appended to every region in each round
