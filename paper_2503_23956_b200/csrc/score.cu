@@ -204,9 +204,11 @@ __device__ __forceinline__ void tile_mma(float (&acc)[4], const KeyFrag<D> &f, c
 // Copies up to 8*NT elite query rows (starting at row0) of one KV group into shared memory, zero padded.
 template <int D>
 __device__ __forceinline__ void stage_queries(uint16_t *s_q, const ScoreParams &p, int grp, int lb, int g,
-                                              int row0, int n_rows_total, int rows_pad) {
+                                              int row0, int n_rows_total, int rows_pad,
+                                              const int32_t *staged_info = nullptr) {
     constexpr int QS = D + 32;
-    const int32_t *info = p.row_info + (int64_t)grp * p.cap;
+    // (head, slot) words of the rows: from the caller's copy in shared memory (rows row0.., row0 = 0) if it has one
+    const int32_t *info = staged_info ? staged_info - row0 : p.row_info + (int64_t)grp * p.cap;
     const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * D;
     for (int idx = threadIdx.x; idx < rows_pad * (D / 8); idx += blockDim.x) {
         const int r = idx / (D / 8), c = idx % (D / 8);
@@ -344,6 +346,12 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     constexpr int QS = D + 32;
     __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
     __shared__ float2 s_stat[NT * 8];  // (row max, weight / normaliser)
+    // the row tables of all KV heads of the sequence, fetched in one go at the start: per head the first NT * 8
+    // rows' (head, slot) words and statistics, so that the loop over the heads waits for the query rows only
+    constexpr int kMaxKv = 8;
+    __shared__ int s_rows[kMaxKv];
+    __shared__ int32_t s_info_all[kMaxKv][NT * 8];
+    __shared__ float2 s_stat_all[kMaxKv][NT * 8];
 
     const int lb = blockIdx.y;
     const int l = lb / p.B, b = lb % p.B;
@@ -351,10 +359,20 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     const int kbase = blockIdx.x * kScoreKeyTile + warp * 32;
     float imp[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [m-tile][key gid / gid+8]
 
+    for (int i = threadIdx.x; i < p.Hkv * NT * 8; i += blockDim.x) {
+        const int g = i / (NT * 8), r = i % (NT * 8);
+        const int64_t at = (int64_t)(lb * p.Hkv + g) * p.cap + r;
+        const bool inside = r < p.cap;
+        s_info_all[g][r] = inside ? p.row_info[at] : 0;
+        s_stat_all[g][r] = inside ? p.row_final[at] : make_float2(0.f, 0.f);
+        if (r == 0) s_rows[g] = p.row_count[lb * p.Hkv + g];
+    }
+    __syncthreads();
+
     for (int g = 0; g < p.Hkv; ++g) {
         const int grp = lb * p.Hkv + g;
         const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
-        const int n_rows = p.row_count[grp];
+        const int n_rows = s_rows[g];
         KeyFrag<D> f[2];
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
@@ -365,9 +383,10 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
         for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
             const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
             __syncthreads();
-            stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
+            stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8, row0 == 0 ? s_info_all[g] : nullptr);
             for (int r = threadIdx.x; r < nt_used * 8; r += blockDim.x)
-                s_stat[r] = row0 + r < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + r] : make_float2(0.f, 0.f);
+                s_stat[r] = row0 + r >= n_rows ? make_float2(0.f, 0.f)
+                            : (row0 == 0 ? s_stat_all[g][r] : p.row_final[(int64_t)grp * p.cap + row0 + r]);
             __syncthreads();
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
