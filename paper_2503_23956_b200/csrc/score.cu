@@ -175,6 +175,10 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
 // (read straight from global memory) and for the query rows (shared memory).  A dot product does not
 // depend on the order of its terms' indices as long as both operands use the same order.
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void prefetch_l2(const void *ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr) : "memory");
+}
+
 template <int D>
 struct KeyFrag {
     uint4 lo[D / 32];  // key row gid
@@ -265,6 +269,11 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
             const int ka = kt + gid, kb = kt + gid + 8;
             const bool va = ka < key1, vb = kb < key1;
             if (kt + 64 < key1) fetch(f_next, kt + 64);
+            // and the tile after that is asked into L2 (one 128-byte line per lane: 16 rows x D channels)
+            if (kt + 128 < key1 && lane < 16 * (D * 2 / 128)) {
+                const int kp = min(kt + 128 + lane / (D * 2 / 128), key1 - 1);
+                prefetch_l2(k_g + (int64_t)kp * p.s_token + (lane % (D * 2 / 128)) * 64);
+            }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 if (nt < nt_used) {
