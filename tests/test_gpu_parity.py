@@ -106,6 +106,23 @@ def test_score_parity(oracle, case, alpha):
     assert err <= TOL, err
 
 
+@pytest.mark.parametrize("case", ["kv2", "s7b", "g16"])
+def test_score_parity_many_elite_rows_below_the_dense_threshold(oracle, case):
+    """A small but non-zero threshold makes almost every candidate elite (hundreds of rows per KV group on the
+    widest window) while the launch stays on the sparse-window kernels: their loops over slabs of rows run more
+    than once, and the wide instantiation of the statistics pass does the work."""
+    wl = CASES[case]
+    alpha = 1e-4
+    ref = oracle_path(oracle, wl, alpha=alpha)
+    rows = [bin(int(m)).count("1") for m in ref["mask"].ravel()]
+    assert max(rows) * wl.group > 64 or case != "kv2"      # the case is what it claims to be
+    gp = make_gpu(wl, ref)
+    gp.score(ref["qw"].to(DEV), alpha=alpha)
+    assert gp.status() == 0
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"]), "elite sets differ"
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+
+
 @pytest.mark.parametrize("alpha", [0.9, 0.0])
 @pytest.mark.parametrize("layout", ["head_major", "layer_innermost"])
 def test_score_parity_other_cache_layouts(oracle, alpha, layout):
