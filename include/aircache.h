@@ -229,8 +229,9 @@ int aircache_decode_step(const aircache_shape_t *shape, aircache_ragged_t *cache
  * never calls cudaMalloc, cudaFree or any other allocating routine.
  *
  *   Arguments as in aircache_decode_attn, without the workspace.
- *   Limit.   2 * min(SMs, 256) * Hq * (d + 2) * 4 + 7936 bytes must fit in the array
- *            (on a 148-SM B200: Hq * (d + 2) <= 10620, e.g. 64 heads of 128);
+ *   Limit.   7424 + 2 * min(SMs, 256) * 4 * (Hq * (d + 2) rounded up to a multiple of 4)
+ *            bytes must fit in the array (7424 = 256 bytes of status + 1792 tickets;
+ *            on a 148-SM B200: Hq * (d + 2) <= 10620, e.g. 80 heads of 128);
  *            larger problems get AIRCACHE_ERR_STATIC_SCRATCH and nothing is enqueued.
  *   Set-up.  The first call on each device looks up the array's device address
  *            (with that device current).  Make that first call before any

@@ -18,8 +18,11 @@ namespace {
 constexpr int kSelThreads = 512;
 constexpr int kSelSmemKeys = 40960;  // scores kept in shared memory up to this many visual tokens
 
+// Order-preserving integer image of a float: a > b as floats <=> key(a) > key(b), a == b <=> equal keys.  The
+// two zeros compare equal as floats, so -0.0 takes the key of +0.0 (the lower index then wins among them).
 __device__ __forceinline__ uint32_t order_key(float x) {
-    const uint32_t u = __float_as_uint(x);
+    uint32_t u = __float_as_uint(x);
+    if ((u << 1) == 0u) u = 0u;
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 

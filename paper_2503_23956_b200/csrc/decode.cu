@@ -43,29 +43,6 @@ namespace aircache {
 
 namespace {
 
-// Development aid, compiled out unless AIRCACHE_DECODE_TRACE is defined: thread 0 of every CTA stores
-// %globaltimer at a few points of the kernel into the unused tail of the partial slots.
-#ifdef AIRCACHE_DECODE_TRACE
-#define DECODE_TRACE(idx)                                                                                   \
-    do {                                                                                                    \
-        if (threadIdx.x == 0) {                                                                             \
-            unsigned long long _t;                                                                          \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));                                          \
-            reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 24 + (idx)] = _t; \
-        }                                                                                                   \
-    } while (0)
-// the same from whichever thread runs it (the producer lane)
-#define DECODE_TRACE_ANY(idx)                                                                               \
-    do {                                                                                                    \
-        unsigned long long _t;                                                                              \
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));                                              \
-        reinterpret_cast<unsigned long long *>(p.partials + (size_t)400 * partial_slot_floats(p.Hq, D))[blockIdx.x * 24 + (idx)] = _t; \
-    } while (0)
-#else
-#define DECODE_TRACE(idx) do { } while (0)
-#define DECODE_TRACE_ANY(idx) do { } while (0)
-#endif
-
 struct DecodeParams {
     const uint16_t *q;       // [L*B, Hq, D]
     float *out;              // [L*B, Hq, D]
@@ -402,7 +379,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     using C = DecodeCfg<D, HKV, G_HI, HS>;
     constexpr int KSPLIT = C::KSPLIT, CH = C::CH, NCW = C::NCW, NROW = C::NROW, kStages = C::NSTAGE;
 
-    DECODE_TRACE(0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *s_stage = smem;
@@ -510,7 +486,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         for (int pass = few ? 0 : 1; pass < 2; ++pass) {
             if (pass) {
                 asm volatile("griddepcontrol.wait;" ::: "memory");
-                DECODE_TRACE(16);
                 if (!few) break;
             }
             rc = plan_few_regions<kPlanRpl, !HS>(
@@ -530,7 +505,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             upc = max(1, small_div(total + n_ctas - 1, n_ctas));
         }
     }
-    DECODE_TRACE(12);
     if (!planned) {
         // ---- unit prefix and first row of all regions (every CTA computes the same tables) ----
         {
@@ -543,7 +517,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
             s_part[tid] = local;
             __syncthreads();
-            DECODE_TRACE(12);
             if (wid == 0) {
                 // warp 0 turns s_part into an exclusive prefix
                 constexpr int PER_LANE = (C::THREADS + 31) / 32;
@@ -574,7 +547,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             if (n == 0 && tid == 0) s_P[0] = 0;
             __syncthreads();
         }
-        DECODE_TRACE(13);
         total = s_P[n];
         upc = max(1, small_div(total + n_ctas - 1, n_ctas));
 
@@ -630,7 +602,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             if (lane == 0) s_aligned = found ? 1 : 0;
         }
         __syncthreads();
-        DECODE_TRACE(14);
         aligned = s_aligned != 0;
 
         // an item without rows yields zeros - or, when a token is appended, that token's value (softmax over one key)
@@ -668,7 +639,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
     }
     if (u0 >= u1) { finish(true); return; }
-    DECODE_TRACE(1);
     // CTAs that hold a piece of region r, and the partial slot CTA c uses for it
     auto span_of = [&](int r, int &c0, int &c1) {
         if (aligned) { c0 = s_Q[r]; c1 = s_Q[r + 1] - 1; }
@@ -706,7 +676,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         tma_load_3d(dst + C::KV_BYTES + off, &tm_v, hf * 64, head, row0, full);
                     }
                 }
-                if (it == 0) DECODE_TRACE_ANY(17);
             }
             if (!ok) {
                 // drain: wait (bounded) for the loads already in flight before the CTA may exit
@@ -737,7 +706,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const int gid = lane >> 2, t = lane & 3;
     const int G = p.G;
 
-    int n_flush = 0;  // flushes done so far (trace slots only)
     int len = 0;      // rows of the item being processed
     // The block's products are taken transposed - S^T = K Q^T and O^T = V^T P^T - so that the 16 rows of the tensor
     // core tile are keys (respectively channels) and its 8 columns the query heads of the KV group: a group of up
@@ -998,7 +966,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 if (s_last) __threadfence();
             }
             consumer_bar(NCW * 32);
-            DECODE_TRACE(4 + 3 * n_flush);
             if (s_last) {
                 if (tid == 0) p.tickets[r] = 0;   // ready for the next call
                 const size_t slot_floats = (size_t)partial_slot_floats(p.Hq, D);
@@ -1057,7 +1024,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                                       slot_bytes, bar);
                     }
                     if (mbar_wait(bar, 0, &s_abort, p.status, 3)) {
-                        DECODE_TRACE(9);
                         const float *sp = reinterpret_cast<const float *>(s_stage);
                         float *wgt = s_merge;   // [np][Hq] weights exp2(m_c - M) / sum
 #pragma unroll 1
@@ -1075,7 +1041,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                                 wgt[c * p.Hq + h] = exp2_or_zero(sp[c * slot_floats + p.Hq * D + h], M) * inv;
                         }
                         consumer_bar(NCW * 32);
-                        DECODE_TRACE(10);
 #pragma unroll 1
                         for (int i = tid; i < items; i += NCW * 32) {
                             const int h = (i * 4) / D;
@@ -1143,15 +1108,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         tok = load_token(r);
         tok_ready = true;
     }
-    DECODE_TRACE(18);
     int it = 0;
     bool ok = true;
     for (int u = u0; u < u1; ++u, ++it) {
         if (u >= s_P[r + 1]) {
-            DECODE_TRACE(3 + 3 * n_flush);
             flush(r, seg_start, u);
-            DECODE_TRACE(5 + 3 * n_flush);
-            n_flush = n_flush < 2 ? n_flush + 1 : 2;
             while (u >= s_P[r + 1]) ++r;
             seg_start = u;
             len = p.lens[r / hs];
@@ -1160,7 +1121,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int s = it % kStages;
         ok = mbar_wait(smem_u32(&s_bar[s]), (it / kStages) & 1, &s_abort, p.status, 2);
         if (!ok) break;
-        if (it == 0) DECODE_TRACE(2);
         const int j0 = (u - s_P[r]) * CH + ks * 16;  // first row of this warp's block inside the region
         if (j0 < len) {
             const uint32_t k_base = smem_u32(s_stage + s * C::STAGE_BYTES) + g * C::HALVES * C::SUBTILE;
@@ -1169,12 +1129,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_bar[kStages + s]));
     }
-    DECODE_TRACE(3 + 3 * n_flush);
     if (ok) flush(r, seg_start, u1);
     if (r_own < 0) finish(false);   // (else the producer warp has drawn the ticket already)
-    DECODE_TRACE(5 + 3 * n_flush);
-    DECODE_TRACE(15);
-    (void)n_flush;
 }
 
 // ---------------------------------------------------------------------------------------------

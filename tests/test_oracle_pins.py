@@ -382,6 +382,13 @@ def test_select_equal_scores_and_planted_subset(oracle_mod):
     assert oracle_mod.select(s, 411).tolist() == want.tolist()
     assert oracle_mod.select(s, 0).tolist() == []
     assert oracle_mod.select(s, 3000).tolist() == list(range(3000))
+    # the two zeros are one value: among them the lower index wins whatever the sign (float comparison, as in
+    # the library's stable sort on the values)
+    assert oracle_mod.select(np.array([-0.0, 0.0, -0.0, 0.0], np.float32), 2).tolist() == [0, 1]
+    z = np.where(rng.integers(0, 2, 400) == 1, np.float32(-0.0), np.float32(0.0)).astype(np.float32)
+    z[rng.choice(400, 60, replace=False)] = rng.choice(np.array([1e-42, -1e-42, 0.5, -0.5], np.float32), 60)
+    want = np.sort(np.lexsort((np.arange(400), -z))[:150])
+    assert oracle_mod.select(z, 150).tolist() == want.tolist()
 
 
 # ----------------------------------------------------------------------------------------------
