@@ -2,24 +2,27 @@
 """Benchmark of the AirCache compress-then-decode hot path on B200.
 
 One *step* is one pass of the whole path over one batch of synthetic requests: for every resident request
-the compression (aircache_score -> aircache_budget -> aircache_compact over all layers), then `decode_steps`
-rounds of single-token decode attention (aircache_decode_attn over all layers) with a fresh query per round.
-`rotate` independent requests (different seeds) are resident and are served round-robin, so that consecutive
-decode launches never find their cache in L2: the per-launch working set of one request at 10 % retention
-(49 MB) is smaller than the 126 MB L2, the rotation makes every launch read HBM as it would between the
-layers of a real model.
+batch the compression (aircache_score -> aircache_budget -> aircache_compact over all layers), then
+`decode_steps` rounds of single-token decode attention (aircache_decode_attn over all layers) with a fresh query
+per round.  `rotate` independent request batches (different seeds) are resident and are served round-robin, so
+that consecutive decode launches never find their cache in L2.
+
+The default workload is the largest one at 10 % visual retention: config 3 (7B shapes, 2916 visual + 256 text
+tokens per sequence) at batch 64, 2 GB of compressed cache per decode launch, 256 decode rounds.
 
   value           tokens / s over the whole step (compression included), inputs resident in HBM
   decode_tok_s    tokens / s over the decode region of the step alone
-  compress_us_per_layer   (score + budget + compact) / layers, per request
+  compress_us_per_layer   (score + budget + compact) / layers, per request batch
   roofline        decode attention: algorithmic bytes (every valid K' and V' row once, q and output) per
                   call / average duration of a call inside the timed region
+  roofline_compact, roofline_score   the same for aircache_compact and aircache_score
   e2e             the same metric through aircache_pipeline_host: pinned host inputs, host outputs
   cpu_baseline    the CPU oracle timed on this host (rank 0, N = 1 only)
   allocation_ablation   budget vectors of the four allocation rules (mode flag) and their JS divergence
-  hbm_bound_workloads   the decode and compaction rooflines on further workloads (default: config 4, 261 MB
-                  per decode launch, and config 3 at batch 16 and 64, 0.5 and 2 GB per launch), measured briefly
-                  after the main run at N = 1
+  workloads       every other configuration and sweep point (config 2 at 50 / 25 / 10 / 5 % retention - at 10 %
+                  also with the cache resident in L2 and without CUDA graphs -, config 3 at batch 1 / 8 / 32,
+                  config 4, config 5) with its full number of decode rounds, measured briefly after the main
+                  run at N = 1: stage times, the three rooflines, clocks
 
 `python bench.py --impl reference` times the CPU oracle instead (there is no other implementation of the
 paper's method to run).  Under torchrun every rank runs the same workload on its own GPU with its own seeds
@@ -46,10 +49,13 @@ import torch  # noqa: E402
 METRIC = "decode_tok_s_at_10pct_visual_kv"
 UNIT = "tok/s"
 L2_BYTES = 126 * 2 ** 20
+Q_RING, O_RING = 16, 8
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from the ncu capture summarised
-# in profiles/; valid only for the kernel source it was taken on (sha1 of csrc/decode.cu, first 12 hex).
-NCU_TRAFFIC = {"workload": "c2", "decode_cu_sha1": "c37c1ce85fef", "bytes_per_launch": 49489000}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from an ncu capture (config 3 at
+# batch 16, the largest case the capture rules allow; traffic grows in proportion to the rows, so it is scaled
+# to the launch that was timed).  Valid only for the kernel source it was taken on (sha1 of csrc/decode.cu,
+# first 12 hex); null otherwise.
+NCU_TRAFFIC = {"workload": "c3", "decode_cu_sha1": "", "bytes_per_valid_row": None}
 
 
 def parse_args():
@@ -58,25 +64,29 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="c2", help="c1 | c2 | c3[:batch] | c4 | c5")
+    ap.add_argument("--workload", default="c3:64", help="c1 | c2 | c3 | c4 | c5, optionally :batch and @ratio")
     ap.add_argument("--ratio", type=float, default=None)
     ap.add_argument("--alpha", type=float, default=None, help="relevance threshold of Eq. 5 (default 0.9; 0 = dense window)")
     ap.add_argument("--rotate", type=int, default=0, help="resident requests (0 = enough to exceed 2x L2)")
     ap.add_argument("--decode-steps", type=int, default=0, help="decode rounds per step (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every time (no CUDA graph)")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--extra", default="c4,c3:16,c3:64", help="comma list of further workloads measured briefly at N = 1 "
-                                                  "(decode and compaction rooflines); \"none\" to skip")
+    ap.add_argument("--extra", default="c2,c2@0.5,c2@0.25,c2@0.05,c3:1,c3:8,c3:32,c4,c5",
+                    help="comma list of further workloads measured briefly at N = 1 (stage times and rooflines); "
+                         "\"none\" to skip")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
 
 def pick_workload(spec: str, ratio, alpha=None):
     from workloads import CONFIGS
+    spec, _, at = spec.partition("@")
     name, _, arg = spec.partition(":")
     wl = CONFIGS[name]
     if arg:
         wl = wl.with_(batch=int(arg))
+    if at:
+        wl = wl.with_(ratio=float(at))
     if ratio is not None:
         wl = wl.with_(ratio=ratio)
     if alpha is not None:
@@ -195,8 +205,10 @@ def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, ap
         k, v = full_cache(w, "k", dev), full_cache(w, "v", dev)
         s.set_full(logical(k), logical(v))
         s.qw = window_queries(w, dev)
-        s.q_steps = torch.stack([decode_queries(w, t, dev) for t in range(n_dec)]).contiguous()
-        s.out_steps = torch.empty((n_dec,) + tuple(s.out.shape), dtype=torch.float32, device=dev)
+        # the decode rounds cycle through Q_RING distinct query sets and O_RING output buffers (what a round
+        # reads and writes besides the cache is a few KB per region)
+        s.q_steps = torch.stack([decode_queries(w, t, dev) for t in range(min(n_dec, Q_RING))]).contiguous()
+        s.out_steps = torch.empty((min(n_dec, O_RING),) + tuple(s.out.shape), dtype=torch.float32, device=dev)
         reqs.append(s)
     torch.cuda.synchronize()
     stream = torch.cuda.Stream(device=dev)
@@ -216,11 +228,11 @@ def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, ap
     def stage_decode():
         for t in range(n_dec):
             for s in reqs:
+                q, out = s.q_steps[t % Q_RING], s.out_steps[t % O_RING]
                 if append:
-                    ac.aircache_decode_step(s.sh, s.cache, s.q_steps[t], s.k_new[t], s.v_new[t], t, s.out_steps[t],
-                                            s.ws, stream)
+                    ac.aircache_decode_step(s.sh, s.cache, q, s.k_new[t], s.v_new[t], t, out, s.ws, stream)
                 else:
-                    s.decode(s.q_steps[t], out=s.out_steps[t], stream=stream)
+                    s.decode(q, out=out, stream=stream)
 
     stages = [("score", stage_score), ("budget", stage_budget), ("compact", stage_compact), ("decode", stage_decode)]
     graphs = {}
@@ -272,27 +284,33 @@ def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, ap
 
 
 def rooflines(ac, wl, m, rotate, n_dec, traffic=None):
-    """Decode-attention and compaction rooflines from one measurement (algorithmic bytes / measured time)."""
+    """Rooflines of decode attention, compaction and scoring from one measurement (algorithmic bytes /
+    measured time).  Algorithmic bytes: decode - every valid K' and V' row once, the queries and the fp32
+    outputs; compaction - every row of the compressed cache read and written once, plus the kept indices;
+    scoring - every visual key once (the second pass of Eq. 7 is meant to find them in L2) plus the scores."""
     sh = shape_of(ac, wl)
     row_bytes = wl.n_kv_heads * wl.head_dim * 2
     T = ac.aircache_kept_per_sequence(sh, wl.ratio)
-    q_out_bytes = wl.n_layers * wl.batch * wl.n_q_heads * wl.head_dim * 6
+    LB = wl.n_layers * wl.batch
+    q_out_bytes = LB * wl.n_q_heads * wl.head_dim * 6
     alg_bytes = 2 * row_bytes * m["valid_rows"] + q_out_bytes
     call_us = m["stage_ms"]["decode"] * 1e3 / (rotate * n_dec)
-    achieved = alg_bytes / (call_us * 1e-6) / 1e9
     peak, peak_kind = measured_peaks()
+
+    def roof(kernel, nbytes, us, **more):
+        gbs = nbytes / (us * 1e-6) / 1e9
+        return {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peak, "peak_kind": f"of {peak_kind}",
+                "unit": "GB/s", "frac": gbs / peak, "frac_of_8TBs_nominal": gbs / 8000.0, **more,
+                "bytes_per_call": nbytes, "us_per_call": us}
+
+    dec = roof("decode_kernel (one launch per aircache_decode_attn call)", alg_bytes, call_us, traffic=traffic)
     compact_bytes = 2 * alg_bytes - 2 * q_out_bytes + 4 * wl.batch * T     # read + write of every row, indices
-    comp_us = m["stage_ms"]["compact"] * 1e3 / rotate
-    dec = {"kernel": "decode_kernel (one launch per aircache_decode_attn call)", "bound": "hbm",
-           "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-           "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": traffic,
-           "bytes_per_call": alg_bytes, "us_per_call": call_us}
-    comp = {"kernel": "select_kernel + gather_kernel per aircache_compact call", "bound": "hbm",
-            "achieved": compact_bytes / (comp_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-            "frac": compact_bytes / (comp_us * 1e-6) / 1e9 / peak,
-            "frac_of_8TBs_nominal": compact_bytes / (comp_us * 1e-6) / 1e9 / 8000.0,
-            "bytes_per_call": compact_bytes, "us_per_call": comp_us}
-    return dec, comp
+    comp = roof("select_kernel + gather_kernel per aircache_compact call", compact_bytes,
+                m["stage_ms"]["compact"] * 1e3 / rotate)
+    score_bytes = LB * wl.n_visual * (row_bytes + 4)
+    score = roof("elite_kernel + stats_kernel + importance_kernel per aircache_score call", score_bytes,
+                 m["stage_ms"]["score"] * 1e3 / rotate)
+    return dec, comp, score
 
 
 def default_rotate(ac, wl):
@@ -308,6 +326,71 @@ def kernels_per_step(wl, rotate, n_dec):
     nt_max = (wl.group * wl.window + 7) // 8
     score = 1 + (1 if nt_max <= 4 else 2) + 1
     return rotate * (score + 1 + 2 + n_dec)
+
+
+def config_of(ac, wl, n_dec, rotate, graph=True):
+    """The `config` object of the JSON line (the reference arm reports the same one)."""
+    _, cache_bytes = default_rotate(ac, wl)
+    return {"workload": describe(wl), "decode_steps": n_dec, "resident_requests": rotate,
+            "l2": f"inputs larger than L2: {rotate} independent request batches served round-robin, "
+                  f"{rotate * cache_bytes / 2 ** 20:.0f} MiB of compressed cache cycled per decode round",
+            "launch": "CUDA graph replay of the C-ABI calls" if graph else "direct C-ABI calls",
+            "attention_only": True}
+
+
+def decode_only(ac, reqs, n_dec, reps, dev, graph):
+    """Average time (us) of one aircache_decode_attn call over the sessions `reqs` served round-robin, the
+    compressed caches as they stand: `reps` timed passes of n_dec rounds after one untimed pass."""
+    stream = torch.cuda.Stream(device=dev)
+
+    def rounds():
+        for t in range(n_dec):
+            for s in reqs:
+                s.decode(s.q_steps[t % Q_RING], out=s.out_steps[t % O_RING], stream=stream)
+
+    with torch.cuda.stream(stream):
+        g = None
+        if graph:
+            rounds()
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                rounds()
+        run = g.replay if g is not None else rounds
+        for _ in range(2):
+            run()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            run()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * n_dec * len(reqs))
+
+
+def workload_report(ac, spec, dev, rank, use_graph):
+    """One further workload, measured briefly: stage times, the three rooflines, clocks."""
+    w2 = pick_workload(spec, None)
+    r2, _ = default_rotate(ac, w2)
+    d2 = w2.steps
+    m2, q2 = measure(ac, w2, d2, r2, 3, 3, use_graph, dev, rank, None)
+    dec2, comp2, score2 = rooflines(ac, w2, m2, r2, d2)
+    rep = {"workload": describe(w2), "decode_steps": d2, "resident_requests": r2,
+           "decode_tok_s": r2 * d2 * w2.batch / (m2["stage_ms"]["decode"] * 1e-3),
+           "compress_us_per_layer": (m2["stage_ms"]["score"] + m2["stage_ms"]["budget"] +
+                                     m2["stage_ms"]["compact"]) * 1e3 / (r2 * w2.n_layers),
+           "stage_us_per_request": {k: v * 1e3 / r2 for k, v in m2["stage_ms"].items()},
+           "roofline": dec2, "roofline_compact": comp2, "roofline_score": score2, "clocks": m2["clocks"]}
+    if 2 * m2["valid_rows"] * w2.n_kv_heads * w2.head_dim * 2 < L2_BYTES // 2:
+        # The compressed cache of one request fits in L2: the same launch with its cache resident there (one
+        # request, nothing rotated in between) next to the rotated, HBM-fed number above; and the per-call
+        # time without CUDA graphs (tensor maps encoded and the launch configured on every call).
+        warm_us = decode_only(ac, q2[:1], min(d2, 64), 5, dev, use_graph)
+        rep["decode_l2_resident"] = {"us_per_call": warm_us, "cold_us_per_call": dec2["us_per_call"],
+                                     "note": "one resident request: its compressed cache stays in L2 between calls"}
+        rep["decode_no_graph_us_per_call"] = decode_only(ac, q2, min(d2, 64), 3, dev, False)
+    del q2
+    return rep
 
 
 def run_cuda(args):
@@ -336,68 +419,55 @@ def run_cuda(args):
     total_ms_all, tokens_all = reduce_over_ranks(m["total_ms"], tokens_per_step * args.steps, dev, dist)
     decode_ms_all, _ = reduce_over_ranks(stage_ms["decode"], 0, dev, dist)
     traffic = None
-    if NCU_TRAFFIC["bytes_per_launch"] and NCU_TRAFFIC["decode_cu_sha1"] == decode_cu_sha1() \
-            and NCU_TRAFFIC["workload"] == args.workload and args.ratio is None:
-        traffic = NCU_TRAFFIC["bytes_per_launch"]
-    roof_dec, roof_comp = rooflines(ac, wl, m, rotate, n_dec, traffic)
+    if NCU_TRAFFIC["bytes_per_valid_row"] and NCU_TRAFFIC["decode_cu_sha1"] == decode_cu_sha1() \
+            and args.workload.startswith(NCU_TRAFFIC["workload"]):
+        traffic = NCU_TRAFFIC["bytes_per_valid_row"] * m["valid_rows"]
+    roof_dec, roof_comp, roof_score = rooflines(ac, wl, m, rotate, n_dec, traffic)
 
     result = {
         "metric": METRIC, "value": tokens_all / (total_ms_all * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": warmup, "ms_per_step": total_ms_all / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": describe(wl), "decode_steps": n_dec, "resident_requests": rotate,
-                   "l2": f"inputs larger than L2: {rotate} independent requests served round-robin, "
-                         f"{rotate * cache_bytes / 2 ** 20:.0f} MiB of compressed cache cycled per decode round",
-                   "launch": "CUDA graph replay of the C-ABI calls" if m["graph"] else "direct C-ABI calls",
-                   "attention_only": True},
+        "config": config_of(ac, wl, n_dec, rotate, m["graph"]),
         "decode_tok_s": world * tokens_per_step / (decode_ms_all * 1e-3),
         "compress_us_per_layer": (stage_ms["score"] + stage_ms["budget"] + stage_ms["compact"]) * 1e3
                                  / (rotate * wl.n_layers),
         "stage_us_per_request": {k: v * 1e3 / rotate for k, v in stage_ms.items()},
         "roofline": roof_dec,
         "roofline_compact": roof_comp,
+        "roofline_score": roof_score,
         "clocks": m["clocks"],
         "gpu_launches": args.steps * kernels_per_step(wl, rotate, n_dec),
     }
     if rank == 0 and not args.no_e2e:
-        result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 5))
+        result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 3))
     if rank == 0 and world == 1 and args.extra not in ("", "none"):
         result["allocation_ablation"] = allocation_ablation(ac, wl, reqs[0])
-        result["score_dense_window"] = dense_window_score(wl, reqs[0])
     del reqs
     torch.cuda.empty_cache()
 
-    # The default workload moves 49 MB per decode launch, about 7.6 us of HBM time: launch, prologue and the
-    # split-K merge weigh as much as the stream.  The same kernels on the HBM-bound configurations:
+    # every other configuration and sweep point, briefly
     if rank == 0 and world == 1 and args.extra not in ("", "none"):
         extra = {}
         for spec in args.extra.split(","):
             try:
-                w2 = pick_workload(spec, None)
-                r2, _ = default_rotate(ac, w2)
-                d2 = min(w2.steps, 32)
-                m2, q2 = measure(ac, w2, d2, r2, 3, 3, not args.no_graph, dev, rank, None)
-                dec2, comp2 = rooflines(ac, w2, m2, r2, d2)
-                extra[spec] = {"workload": describe(w2), "decode_steps": d2, "resident_requests": r2,
-                               "decode_tok_s": r2 * d2 * w2.batch / (m2["stage_ms"]["decode"] * 1e-3),
-                               "compress_us_per_layer": (m2["stage_ms"]["score"] + m2["stage_ms"]["budget"] +
-                                                         m2["stage_ms"]["compact"]) * 1e3 / (r2 * w2.n_layers),
-                               "stage_us_per_request": {k: v * 1e3 / r2 for k, v in m2["stage_ms"].items()},
-                               "roofline": dec2, "roofline_compact": comp2, "clocks": m2["clocks"]}
-                del q2
+                extra[spec] = workload_report(ac, spec, dev, rank, not args.no_graph)
             except torch.cuda.OutOfMemoryError as e:
                 # a further workload that does not fit this GPU's free memory does not take the main line down
                 extra[spec] = {"skipped": f"out of device memory: {str(e)[:120]}"}
             torch.cuda.empty_cache()
-        result["hbm_bound_workloads"] = extra
-        # Eq. 2: the same decode rounds with one new token's K/V appended to every region in each round
+        result["workloads"] = extra
+        # config 2: the dense window (alpha = 0, tcgen05) and the decode rounds with the append of Eq. 2 fused in
         # (the cache grows over the rounds: lens change with every launch)
-        d3 = min(n_dec, 64)
-        m3, q3 = measure(ac, wl, d3, rotate, 3, 3, not args.no_graph, dev, rank, None, append=True)
+        w2 = pick_workload("c2", None)
+        r2, _ = default_rotate(ac, w2)
+        d3 = min(w2.steps, 64)
+        m3, q3 = measure(ac, w2, d3, r2, 3, 3, not args.no_graph, dev, rank, None, append=True)
         result["decode_with_append"] = {
-            "decode_steps": d3, "tok_s": rotate * d3 * wl.batch / (m3["stage_ms"]["decode"] * 1e-3),
-            "us_per_round": m3["stage_ms"]["decode"] * 1e3 / (rotate * d3),
+            "workload": describe(w2), "decode_steps": d3, "tok_s": r2 * d3 * w2.batch / (m3["stage_ms"]["decode"] * 1e-3),
+            "us_per_round": m3["stage_ms"]["decode"] * 1e3 / (r2 * d3),
             "note": "aircache_decode_step (Eq. 2 append fused into the attention launch) per round and request"}
+        result["score_dense_window"] = dense_window_score(w2, q3[0])
         del q3
         torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -472,17 +542,25 @@ def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
     k_tm = s.k_full.permute(0, 1, 3, 2, 4)      # back to the token-major storage order
     v_tm = s.v_full.permute(0, 1, 3, 2, 4)
     assert k_tm.is_contiguous()
-    h_k, h_v = k_tm.cpu().pin_memory(), v_tm.cpu().pin_memory()
+    def pinned_copy(t):
+        h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        h.copy_(t)
+        return h
+
+    h_k, h_v = pinned_copy(k_tm), pinned_copy(v_tm)
     h_full = ac.full_view(logical(h_k), logical(h_v))
     d_k, d_v = torch.empty_like(k_tm), torch.empty_like(v_tm)
-    h_qw, h_q = s.qw.cpu().pin_memory(), s.q_steps.cpu().pin_memory()
-    d_qw, d_q = torch.empty_like(s.qw), torch.empty_like(s.q_steps)
-    h_out = torch.empty(s.out_steps.shape, dtype=torch.float32).pin_memory()
-    h_bud = torch.empty(s.budgets.shape, dtype=torch.int32).pin_memory()
+    q_all = s.q_steps[torch.arange(n_dec, device=dev) % s.q_steps.shape[0]]      # [n_dec, L, B, Hq, d]
+    h_qw, h_q = pinned_copy(s.qw), pinned_copy(q_all)
+    d_qw, d_q = torch.empty_like(s.qw), torch.empty_like(q_all)
+    del q_all
+    d_out = torch.empty((n_dec,) + tuple(s.out.shape), dtype=torch.float32, device=dev)
+    h_out = torch.empty(d_out.shape, dtype=torch.float32, pin_memory=True)
+    h_bud = torch.empty(s.budgets.shape, dtype=torch.int32, pin_memory=True)
 
     def once():
         ac.aircache_pipeline_host(sh, h_full, h_k.numel(), d_k, d_v, h_qw, d_qw, h_q, d_q, n_dec, wl.alpha,
-                                  wl.ratio, 0, s.scores, s.budgets, s.cache, s.out_steps, h_out, h_bud, s.ws, stream)
+                                  wl.ratio, 0, s.scores, s.budgets, s.cache, d_out, h_out, h_bud, s.ws, stream)
 
     once()
     torch.cuda.synchronize()
@@ -503,57 +581,80 @@ def run_e2e(ac, wl, sh, s, n_dec, dev, steps):
 # --------------------------------------------------------------------------------------------------
 # the CPU oracle, timed as it stands (cpu_baseline leg and --impl reference)
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(wl, n_dec, max_seqs=1, dec_rounds=4):
-    """Times the oracle on a bounded sample of the workload: the whole compression of `max_seqs` sequences
-    (all layers) and `dec_rounds` decode rounds over their compressed caches; returns seconds."""
-    import oracle
-    from workloads import decode_queries, full_cache, window_queries
-    from workloads.synth import to_u16
-    oracle.build()
-    seqs = list(range(min(max_seqs, wl.batch)))
-    w1 = wl.with_(batch=len(seqs))
-    dm = oracle.Dims(w1.n_layers, w1.batch, w1.n_q_heads, w1.n_kv_heads, w1.head_dim, w1.n_visual, w1.n_text,
-                     w1.window)
-    k, v = full_cache(wl, "k", "cpu", seqs=seqs), full_cache(wl, "v", "cpu", seqs=seqs)
-    qw = window_queries(wl, "cpu", seqs=seqs)
-    kl, vl = to_u16(k).transpose(0, 1, 3, 2, 4), to_u16(v).transpose(0, 1, 3, 2, 4)
-    t0 = time.perf_counter()
-    sc = oracle.score(dm, kl, to_u16(qw), wl.scale, wl.alpha)
-    st, sk = oracle.moments(sc["scores"])
-    bud = oracle.allocate(st, sk, wl.n_visual, wl.ratio, 0)
-    cp = oracle.compact(dm, 0, kl, vl, sc["scores"], bud)
-    t_comp = time.perf_counter() - t0
-    qs = [to_u16(decode_queries(wl, t, "cpu", seqs=seqs)) for t in range(dec_rounds)]
-    t0 = time.perf_counter()
-    for q in qs:
-        oracle.decode(dm, cp["k"], cp["v"], cp["offsets"], cp["lens"], q, wl.scale)
-    t_dec = (time.perf_counter() - t0) / dec_rounds
-    # scale to the whole batch: sequences are independent, the oracle's cost is linear in them
-    f = wl.batch / len(seqs)
-    return {"t_compress": t_comp * f, "t_decode_round": t_dec * f, "threads": oracle.num_threads(),
-            "sample": f"oracle on {len(seqs)} of {wl.batch} sequence(s), all {wl.n_layers} layers: whole compression "
-                      f"once + {dec_rounds} decode rounds; scaled linearly to the batch and to {n_dec} rounds"}
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: `max_seqs` sequences (all layers) and `dec_rounds`
+    decode rounds over their compressed caches.  Inputs are generated once; run() times the oracle."""
+
+    def __init__(self, wl, max_seqs=1, dec_rounds=16):
+        import oracle
+        from workloads import decode_queries, full_cache, window_queries
+        from workloads.synth import to_u16
+        oracle.build()
+        self.oracle, self.wl = oracle, wl
+        self.seqs = list(range(min(max_seqs, wl.batch)))
+        w1 = wl.with_(batch=len(self.seqs))
+        self.dm = oracle.Dims(w1.n_layers, w1.batch, w1.n_q_heads, w1.n_kv_heads, w1.head_dim, w1.n_visual,
+                              w1.n_text, w1.window)
+        k, v = full_cache(wl, "k", "cpu", seqs=self.seqs), full_cache(wl, "v", "cpu", seqs=self.seqs)
+        self.kl, self.vl = to_u16(k).transpose(0, 1, 3, 2, 4), to_u16(v).transpose(0, 1, 3, 2, 4)
+        self.qw = to_u16(window_queries(wl, "cpu", seqs=self.seqs))
+        self.qs = [to_u16(decode_queries(wl, t, "cpu", seqs=self.seqs)) for t in range(dec_rounds)]
+
+    def run(self, n_dec):
+        """Seconds for the whole batch and n_dec rounds, scaled linearly from the sample (sequences are
+        independent and decode rounds alike, so the oracle's cost is linear in both)."""
+        oracle, wl, dm = self.oracle, self.wl, self.dm
+        t0 = time.perf_counter()
+        sc = oracle.score(dm, self.kl, self.qw, wl.scale, wl.alpha)
+        st, sk = oracle.moments(sc["scores"])
+        bud = oracle.allocate(st, sk, wl.n_visual, wl.ratio, 0)
+        cp = oracle.compact(dm, 0, self.kl, self.vl, sc["scores"], bud)
+        t_comp = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        for q in self.qs:
+            oracle.decode(dm, cp["k"], cp["v"], cp["offsets"], cp["lens"], q, wl.scale)
+        t_dec = (time.perf_counter() - t0) / len(self.qs)
+        f = wl.batch / len(self.seqs)
+        return {"t_compress": t_comp * f, "t_decode_round": t_dec * f, "threads": oracle.num_threads(),
+                "sample": f"oracle on {len(self.seqs)} of {wl.batch} sequence(s), all {wl.n_layers} layers: whole "
+                          f"compression once + {len(self.qs)} decode rounds; scaled linearly to the batch and to "
+                          f"{n_dec} rounds"}
 
 
 def cpu_baseline(wl, n_dec):
-    s = oracle_sample(wl, n_dec)
+    s = OracleSample(wl).run(n_dec)
     step_s = s["t_compress"] + n_dec * s["t_decode_round"]
     return {"value": n_dec * wl.batch / step_s, "unit": UNIT, "cores": s["threads"], "kind": "oracle",
-            "sample": s["sample"], "compress_us_per_layer": s["t_compress"] * 1e6 / (wl.n_layers * wl.batch),
+            "sample": s["sample"], "compress_us_per_layer": s["t_compress"] * 1e6 / wl.n_layers,
             "decode_tok_s": wl.batch / s["t_decode_round"]}
+
+
+class _HostArithmetic:
+    """The two host-side numbers config_of() needs, without the CUDA library (the reference arm runs without it)."""
+
+    @staticmethod
+    def shape(*a):
+        return a
+
+    @staticmethod
+    def aircache_kept_per_sequence(sh, ratio):
+        n_layers, n_visual = sh[0], sh[5]
+        return int(np.floor(ratio * float(n_visual * n_layers) + 0.5))
 
 
 def run_reference(args):
     rank, _, world = dist_info()
     if rank != 0:
         return
-    wl = pick_workload(args.workload, args.ratio)
+    wl = pick_workload(args.workload, args.ratio, args.alpha)
     n_dec = args.decode_steps or wl.steps
+    rotate = args.rotate or default_rotate(_HostArithmetic, wl)[0]
+    sample = OracleSample(wl)
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(wl, n_dec, dec_rounds=1)
+        sample.run(n_dec)
     times, last = [], None
     for _ in range(args.steps):
-        last = oracle_sample(wl, n_dec, dec_rounds=2)
+        last = sample.run(n_dec)
         times.append(last["t_compress"] + n_dec * last["t_decode_round"])
     step_s = sum(times) / len(times)
     value = n_dec * wl.batch / step_s
@@ -561,7 +662,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": describe(wl), "decode_steps": n_dec, "attention_only": True},
+        "config": config_of(_HostArithmetic, wl, n_dec, rotate, not args.no_graph),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["threads"], "kind": "oracle",
                          "sample": last["sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

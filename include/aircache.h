@@ -156,6 +156,23 @@ int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, c
                    void *cuda_stream);
 
 /*
+ * Algorithm 1, first loop, a range of its iterations: aircache_score for layers
+ * layer_begin .. layer_begin + layer_count - 1 only.  The paper scores layer by
+ * layer and keeps every layer's full cache until all are scored (Section 4.1
+ * and the limitation noted in Appendix A); an engine calls this at the end of
+ * each layer's prefill, while that layer's keys are still in L2, and runs
+ * aircache_budget once after the last layer.  All arrays are the ones
+ * aircache_score takes (indexed by absolute layer); only the given layers' keys
+ * and window queries are read and only their rows of scores / elite_mask are
+ * written.  The result for a layer is bit-identical to what aircache_score
+ * gives for it, whatever the split into ranges.  Calls that share a workspace
+ * must be ordered on one stream.  layer_count = 0 is a no-op.
+ */
+int aircache_score_layers(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window,
+                          float alpha, int32_t layer_begin, int32_t layer_count, float *scores,
+                          uint64_t *elite_mask, void *workspace, int64_t workspace_bytes, void *cuda_stream);
+
+/*
  * Section 3.4, Eq. 9-11 and the budget line of Algorithm 1.  Per region:
  * strength s_t = sum of I_v (Eq. 9) and skewness s_k = adjusted Fisher-Pearson
  * coefficient with the sample standard deviation (Eq. 10), both in fp64.  Per

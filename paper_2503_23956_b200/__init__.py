@@ -60,6 +60,8 @@ _SIGNATURES = {
     "aircache_workspace_bytes": (C.c_int64, [C.POINTER(Shape)]),
     "aircache_score": (C.c_int, [C.POINTER(Shape), C.POINTER(Full), C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_int64, C.c_void_p]),
+    "aircache_score_layers": (C.c_int, [C.POINTER(Shape), C.POINTER(Full), C.c_void_p, C.c_float, C.c_int32, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_budget": (C.c_int, [C.POINTER(Shape), C.c_void_p, C.c_double, C.c_int32, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.POINTER(Ragged), C.c_void_p, C.c_int64, C.c_void_p]),
     "aircache_compact": (C.c_int, [C.POINTER(Shape), C.POINTER(Full), C.c_void_p, C.c_void_p, C.c_double,
@@ -174,6 +176,16 @@ def aircache_score(sh, full, q_window, alpha, scores, elite_mask, workspace, str
                               _ptr(workspace), _nbytes(workspace), _stream(stream))
     if check:
         _check("aircache_score", rc)
+    return rc
+
+
+def aircache_score_layers(sh, full, q_window, alpha, layer_begin, layer_count, scores, elite_mask, workspace,
+                          stream=None, check=True) -> int:
+    rc = lib().aircache_score_layers(C.byref(sh), C.byref(full), _ptr(q_window), alpha, layer_begin, layer_count,
+                                     _ptr(scores), _ptr(elite_mask), _ptr(workspace), _nbytes(workspace),
+                                     _stream(stream))
+    if check:
+        _check("aircache_score_layers", rc)
     return rc
 
 

@@ -169,9 +169,9 @@ int64_t aircache_workspace_bytes(const aircache_shape_t *shape) {
     return ws_layout(shape).total;
 }
 
-int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window, float alpha,
-                   float *scores, uint64_t *elite_mask, void *workspace, int64_t workspace_bytes,
-                   void *cuda_stream) {
+int aircache_score_layers(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window,
+                          float alpha, int32_t layer_begin, int32_t layer_count, float *scores,
+                          uint64_t *elite_mask, void *workspace, int64_t workspace_bytes, void *cuda_stream) {
     int rc = check_shape(shape);
     if (rc) return rc;
     if ((rc = check_full(shape, full))) return rc;
@@ -179,8 +179,20 @@ int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, c
     if (((uintptr_t)q_window & 15) || ((uintptr_t)scores & 15) || ((uintptr_t)elite_mask & 7))
         return AIRCACHE_ERR_ALIGNMENT;
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return AIRCACHE_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_count < 0 || layer_begin > shape->n_layers - layer_count)
+        return AIRCACHE_ERR_INVALID_ARG;
     if ((rc = check_ws(shape, workspace, workspace_bytes))) return rc;
-    return launch_score(shape, full, q_window, alpha, scores, elite_mask, workspace, (cudaStream_t)cuda_stream);
+    if (layer_count == 0) return AIRCACHE_OK;
+    return launch_score(shape, full, q_window, alpha, layer_begin, layer_count, scores, elite_mask, workspace,
+                        (cudaStream_t)cuda_stream);
+}
+
+int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window, float alpha,
+                   float *scores, uint64_t *elite_mask, void *workspace, int64_t workspace_bytes,
+                   void *cuda_stream) {
+    if (!shape) return AIRCACHE_ERR_INVALID_ARG;
+    return aircache_score_layers(shape, full, q_window, alpha, 0, shape->n_layers, scores, elite_mask, workspace,
+                                 workspace_bytes, cuda_stream);
 }
 
 int aircache_budget(const aircache_shape_t *shape, const float *scores, double ratio, int32_t mode,

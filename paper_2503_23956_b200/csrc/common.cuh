@@ -115,7 +115,7 @@ inline T *ws_ptr(void *ws, int64_t off) {
 
 // entry points implemented per translation unit
 int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void *q_window, float alpha,
-                 float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st);
+                 int layer_begin, int layer_count, float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st);
 int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, int32_t mode, int32_t *budgets,
                   double *strength, double *skewness, aircache_ragged_t *layout, void *ws, cudaStream_t st);
 int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const float *scores,

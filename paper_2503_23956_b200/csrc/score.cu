@@ -41,6 +41,7 @@ struct ScoreParams {
     float2 *row_final;   // (max, weight / normaliser) per elite row, written by the last stats CTA of a group
     uint32_t *group_ticket;
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
+    int lb0, n_lb;   // the launch covers regions lb0 .. lb0 + n_lb - 1 (a range of layers)
     int cap, chunks, chunk_keys;
     float scale, sl2, ln_alpha;
     int keep_all;
@@ -66,7 +67,7 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     __shared__ uint64_t s_mask[kMaxGroup];
     __shared__ int s_first_row[kMaxGroup + 1];
 
-    const int grp = blockIdx.x;  // (l*B + b)*Hkv + g
+    const int grp = p.lb0 * p.Hkv + blockIdx.x;  // (l*B + b)*Hkv + g
     const int g = grp % p.Hkv;
     const int lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
@@ -234,7 +235,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
     __shared__ float2 s_red[4][NT * 8];
     __shared__ int s_is_last;
 
-    const int grp = blockIdx.y;
+    const int grp = p.lb0 * p.Hkv + blockIdx.y;
     const int g = grp % p.Hkv;
     const int lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
@@ -362,7 +363,7 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
     __shared__ int32_t s_info_all[kMaxKv][NT * 8];
     __shared__ float2 s_stat_all[kMaxKv][NT * 8];
 
-    const int lb = blockIdx.y;
+    const int lb = p.lb0 + blockIdx.y;
     const int l = lb / p.B, b = lb % p.B;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
     const int kbase = blockIdx.x * kScoreKeyTile + warp * 32;
@@ -522,7 +523,7 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
     __shared__ int s_abort, s_is_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int grp = blockIdx.y;
+    const int grp = p.lb0 * p.Hkv + blockIdx.y;
     const int g = grp % p.Hkv, lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
     const int chunk = blockIdx.x;
@@ -651,7 +652,7 @@ __global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_cons
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int lb = blockIdx.y;
+    const int lb = p.lb0 + blockIdx.y;
     const int l = lb / p.B, b = lb % p.B;
     const int key0 = blockIdx.x * 128 * KT;
     const int n_tiles = min(KT, (p.Nv - key0 + 127) / 128);
@@ -742,14 +743,14 @@ __global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_cons
 template <int D, int NT>
 int launch_stats(ScoreParams p, int rows_lo, int rows_hi, cudaStream_t st) {
     p.rows_lo = rows_lo; p.rows_hi = rows_hi;
-    stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)((int64_t)p.L * p.B * p.Hkv)), 128, 0, st>>>(p);
+    stats_kernel<D, NT><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), 128, 0, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }
 
 template <int D, int NT>
 int launch_importance(const ScoreParams &p, cudaStream_t st) {
-    importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)((int64_t)p.L * p.B)), 128, 0,
+    importance_kernel<D, NT><<<dim3((p.Nv + kScoreKeyTile - 1) / kScoreKeyTile, (unsigned)p.n_lb), 128, 0,
                                st>>>(p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
@@ -815,9 +816,9 @@ int launch_dense(ScoreParams &p, const CUtensorMap &tm, cudaStream_t st) {
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_STATS));
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_importance_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            C::SMEM_IMP));
-    dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.L * p.B * p.Hkv)), 128, C::SMEM_STATS, st>>>(tm, p);
+    dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), 128, C::SMEM_STATS, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
-    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)((int64_t)p.L * p.B)), 128,
+    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)p.n_lb), 128,
                                  C::SMEM_IMP, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
@@ -826,7 +827,7 @@ int launch_dense(ScoreParams &p, const CUtensorMap &tm, cudaStream_t st) {
 }  // namespace
 
 int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void *q_window, float alpha,
-                 float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st) {
+                 int layer_begin, int layer_count, float *scores, uint64_t *elite_mask, void *ws, cudaStream_t st) {
     const WsLayout w = ws_layout(s);
     ScoreParams p;
     p.k = (const uint16_t *)f->k;
@@ -843,6 +844,8 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.group_ticket = ws_ptr<uint32_t>(ws, w.group_ticket);
     p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
     p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
+    p.lb0 = layer_begin * s->batch;
+    p.n_lb = layer_count * s->batch;
     p.cap = score_row_cap(s);
     p.chunks = score_chunks(s);
     p.chunk_keys = (int)align_up((s->n_visual + p.chunks - 1) / p.chunks, 16);
@@ -854,7 +857,7 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.pos_token = p.pos_head = p.pos_batch = p.pos_layer = 0;
     p.status = ws_ptr<uint32_t>(ws, w.status);
 
-    const int64_t groups = (int64_t)p.L * p.B * p.Hkv;
+    const int64_t groups = (int64_t)p.n_lb * p.Hkv;
     const size_t elite_smem = (size_t)(p.W + p.G) * (p.d + 8) * 2;
     if (s->head_dim == 64) elite_kernel<64><<<(unsigned)groups, 128, elite_smem, st>>>(p);
     else elite_kernel<128><<<(unsigned)groups, 128, elite_smem, st>>>(p);

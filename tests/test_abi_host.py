@@ -101,6 +101,12 @@ def test_entry_points_reject_bad_arguments_on_the_host():
                              check=False) == ac.ERR_WORKSPACE_TOO_SMALL
     assert ac.aircache_score(sh, full, P, 0.9, P, None, Ws(P + 16, ws_bytes), s, check=False) == ac.ERR_ALIGNMENT
     assert ac.aircache_score(sh, full, P, 0.9, P, None, None, s, check=False) == ac.ERR_INVALID_ARG
+    # score, a range of layers
+    for begin, count in ((-1, 1), (0, 3), (2, 1), (1, 2), (0, -1)):
+        assert ac.aircache_score_layers(sh, full, P, 0.9, begin, count, P, None, ws, s,
+                                        check=False) == ac.ERR_INVALID_ARG, (begin, count)
+    assert ac.aircache_score_layers(sh, full, P, 0.9, 2, 0, P, None, ws, s, check=False) == ac.OK   # empty range
+    assert ac.aircache_score_layers(sh, full, P + 2, 0.9, 0, 1, P, None, ws, s, check=False) == ac.ERR_ALIGNMENT
     # budget
     assert ac.aircache_budget(sh, P, 1.2, 0, P, None, None, rag, ws, s, check=False) == ac.ERR_INVALID_ARG
     assert ac.aircache_budget(sh, P, 0.5, 4, P, None, None, rag, ws, s, check=False) == ac.ERR_INVALID_ARG

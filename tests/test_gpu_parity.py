@@ -353,6 +353,32 @@ def test_full_retention_equals_full_cache_decode(oracle):
     assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
 
 
+@pytest.mark.parametrize("case,alpha", [("s7b", 0.9), ("s7b", 0.0), ("c1", 0.9), ("many", 0.9)])
+def test_scoring_layer_by_layer_equals_one_call(oracle, case, alpha):
+    """Algorithm 1's first loop taken a layer (or a few layers) at a time: aircache_score_layers over any split of
+    the layers writes the same bits as one aircache_score call, and those match the oracle."""
+    import paper_2503_23956_b200 as ac
+    wl = CASES[case]
+    ref = oracle_path(oracle, wl, alpha=alpha)
+    gp = make_gpu(wl, ref)
+    qw = ref["qw"].to(DEV)
+    gp.score(qw, alpha=alpha)
+    whole, whole_mask = gp.scores.clone(), gp.mask.clone()
+    L = wl.n_layers
+    for ranges in ([(l, 1) for l in range(L)], [(0, L // 2), (L // 2, L - L // 2)][::-1]):
+        gp.scores.fill_(float("nan")); gp.mask.fill_(-1)
+        for begin, count in ranges:
+            ac.aircache_score_layers(gp.sh, gp.full, qw, alpha, begin, count, gp.scores, gp.mask, gp.ws)
+        assert gp.status() == 0
+        assert torch.equal(gp.scores, whole) and torch.equal(gp.mask, whole_mask)
+    # a single layer leaves the other layers' rows alone
+    gp.scores.fill_(float("nan"))
+    ac.aircache_score_layers(gp.sh, gp.full, qw, alpha, L - 1, 1, gp.scores, gp.mask, gp.ws)
+    assert torch.isnan(gp.scores[:L - 1]).all() and torch.equal(gp.scores[L - 1], whole[L - 1])
+    assert np.array_equal(whole_mask.cpu().numpy().view(np.uint64), ref["mask"])
+    assert rel_elem_err(whole.cpu().numpy(), ref["scores"]) <= TOL
+
+
 def test_results_are_bit_reproducible(oracle):
     wl = CASES["s7b"]
     ref = oracle_path(oracle, wl)
