@@ -30,7 +30,9 @@
  *             aircache_check_status() and aircache_pipeline_host().
  * Errors.     Return value 0 = success, negative = an AIRCACHE_ERR_* code.  All
  *             argument checks run on the host before anything is launched, so a
- *             failing call has enqueued nothing.  No exception crosses the ABI.
+ *             failing call has enqueued nothing (aircache_pipeline_host, which
+ *             issues many copies and launches, is the exception: see there).
+ *             No exception crosses the ABI.
  * Threads.    The library keeps no mutable global state apart from a per-thread
  *             copy of the last CUDA error code and the device address of the
  *             built-in array of aircache_decode_attn_static (looked up once per
@@ -318,7 +320,11 @@ int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes);
  * d_full_v stays untouched; otherwise V is uploaded whole like K.  The outputs of the
  * decode rounds are copied back in groups of 16 rounds on a second stream that
  * the call creates and destroys, so that the download overlaps the later rounds;
- * on return every copy has completed.
+ * on return every copy has completed.  The call clears the workspace's status
+ * words itself.  If a copy or a launch fails after the first copy has been
+ * enqueued, the call still drains both streams before it returns the error, so
+ * the host buffers are never touched after the return; the device buffers then
+ * hold partial results.
  *   h_full       HOST view of the full cache (strides as in aircache_full_t)
  *   full_elems   elements (bf16) spanned by h_full->k and by h_full->v
  *   d_full_k/v   DEVICE buffers of full_elems bf16 each

@@ -350,6 +350,19 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     if (!(alpha >= 0.0f && alpha <= 1.0f) || !(ratio >= 0.0 && ratio <= 1.0) || mode < 0 || mode > 3)
         return AIRCACHE_ERR_INVALID_ARG;
 
+    // From here on work is in flight on the stream (and later on the copy stream) that reads and writes the
+    // caller's host buffers: whatever happens, the call returns only after both streams have drained.
+    struct CopySide {
+        cudaStream_t main = nullptr, stream = nullptr;
+        cudaEvent_t event = nullptr;
+        ~CopySide() {
+            if (stream) cudaStreamSynchronize(stream);
+            cudaStreamSynchronize(main);
+            if (event) cudaEventDestroy(event);
+            if (stream) cudaStreamDestroy(stream);
+        }
+    } side;
+    side.main = st;
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_k, h_full->k, full_elems * 2, cudaMemcpyHostToDevice, st));
     if (!v_in_place)
         AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_v, h_full->v, full_elems * 2, cudaMemcpyHostToDevice, st));
@@ -357,6 +370,7 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     if (n_steps > 0)
         AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_q_steps, h_q_steps, (int64_t)n_steps * q_elems * 2,
                                           cudaMemcpyHostToDevice, st));
+    if ((rc = aircache_reset_status(workspace, workspace_bytes, st))) return rc;
     if ((rc = aircache_score(shape, &d_full, d_q_window, alpha, d_scores, nullptr, workspace, workspace_bytes, st)))
         return rc;
     if ((rc = aircache_budget(shape, d_scores, ratio, mode, d_budgets, nullptr, nullptr, d_cache, workspace,
@@ -367,14 +381,6 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
         return rc;
     // The results go back to the host while later rounds still run: a second stream copies every
     // kCopyEvery rounds' outputs as soon as the round that wrote the last of them has finished.
-    struct CopySide {
-        cudaStream_t stream = nullptr;
-        cudaEvent_t event = nullptr;
-        ~CopySide() {
-            if (event) cudaEventDestroy(event);
-            if (stream) cudaStreamDestroy(stream);
-        }
-    } side;
     constexpr int32_t kCopyEvery = 16;
     if (n_steps > 0) {
         AIRCACHE_CUDA_TRY(cudaStreamCreateWithFlags(&side.stream, cudaStreamNonBlocking));

@@ -379,6 +379,46 @@ def test_scoring_layer_by_layer_equals_one_call(oracle, case, alpha):
     assert rel_elem_err(whole.cpu().numpy(), ref["scores"]) <= TOL
 
 
+def test_system_prompt_prefix_as_leading_text_rows(oracle):
+    """A system prompt handed over as the leading text rows: it lies outside the last W text rows that Eq. 5 draws
+    its candidates from and outside the softmax of Eq. 7, so the scores, budgets and kept visual tokens are those of
+    the cache without it (however loud its keys), every prefix row is in the compressed cache, and decode attends
+    to it like the oracle does."""
+    wl = CASES["s7b"]
+    P = 24
+    ref = oracle_path(oracle, wl)
+    rng = np.random.default_rng(31)
+    Nv = wl.n_visual
+    shape = (wl.n_layers, wl.batch, P, wl.n_kv_heads, wl.head_dim)
+    pk = torch.from_numpy((rng.standard_normal(shape) * 30.0).astype(np.float32)).to(torch.bfloat16)
+    pv = torch.from_numpy(rng.standard_normal(shape).astype(np.float32)).to(torch.bfloat16)
+    k2 = torch.cat([ref["k"][:, :, :Nv], pk, ref["k"][:, :, Nv:]], dim=2).contiguous()     # token-major storage
+    v2 = torch.cat([ref["v"][:, :, :Nv], pv, ref["v"][:, :, Nv:]], dim=2).contiguous()
+    wl2 = wl.with_(name="s7b_sys", n_text=wl.n_text + P)
+    gp = GpuPath(wl2, ratio=ref["ratio"], device=DEV)
+    gp.set_full(logical(k2.to(DEV)), logical(v2.to(DEV)))
+    gp.score(ref["qw"].to(DEV), alpha=ref["alpha"])
+    gp.budget()
+    gp.compact()
+    assert gp.status() == 0
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"])
+    assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+    assert np.array_equal(gp.budgets.cpu().numpy(), ref["budgets"])
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(ref["compact"]["kept_idx"])], ref["compact"]["kept_idx"])
+    dm2 = oracle_dims(oracle, wl2)
+    cp2 = oracle.compact(dm2, 0, u16(logical(k2)), u16(logical(v2)), ref["scores"], ref["budgets"])
+    compare_cache(gp, cp2)
+    kc = u16(gp.k_c)
+    for r in range(len(cp2["lens"])):
+        l, b = divmod(r, wl.batch)
+        first_text = int(cp2["offsets"][r]) + int(ref["budgets"][l, b])
+        assert np.array_equal(kc[first_text:first_text + P], u16(pk[l, b]))
+    q = decode_queries(wl, 0, "cpu")
+    want = oracle.decode(dm2, cp2["k"], cp2["v"], cp2["offsets"], cp2["lens"], u16(q), wl.scale)
+    gp.decode(q.to(DEV))
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+
+
 def test_results_are_bit_reproducible(oracle):
     wl = CASES["s7b"]
     ref = oracle_path(oracle, wl)

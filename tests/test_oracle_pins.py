@@ -137,6 +137,30 @@ def test_scores_match_matrix_form_and_sum_to_one(oracle_mod, alpha):
         assert abs(s_t - (1 - out["text_mass"][l, b].mean())) < 1e-6
 
 
+def test_system_prompt_prefix_is_kept_and_stays_out_of_the_scores(oracle_mod):
+    """A system prompt passed as leading text rows (Section 3.3: it is left out of the window): the scores are the
+    ones of the same cache without the prefix, whatever the prefix holds, and every prefix row survives compaction
+    in place, in front of the other text rows."""
+    rng = np.random.default_rng(21)
+    L, B, Hq, Hkv, d, Nv, Nt, W, P = 2, 2, 4, 2, 16, 37, 9, 6, 5
+    k, v, qw = rand_case(rng, L, B, Hq, Hkv, d, Nv, Nt, W)
+    prefix_k = bf16_bits(rng.standard_normal((L, B, Hkv, P, d)) * 50.0)   # loud rows: they would show in any softmax
+    prefix_v = bf16_bits(rng.standard_normal((L, B, Hkv, P, d)))
+    k2 = np.concatenate([k[:, :, :, :Nv], prefix_k, k[:, :, :, Nv:]], axis=3)
+    v2 = np.concatenate([v[:, :, :, :Nv], prefix_v, v[:, :, :, Nv:]], axis=3)
+    dm, dm2 = oracle_mod.Dims(L, B, Hq, Hkv, d, Nv, Nt, W), oracle_mod.Dims(L, B, Hq, Hkv, d, Nv, Nt + P, W)
+    a, b2 = oracle_mod.score(dm, k, qw, 0.25, 0.9), oracle_mod.score(dm2, k2, qw, 0.25, 0.9)
+    assert np.array_equal(a["scores"], b2["scores"]) and np.array_equal(a["elite_mask"], b2["elite_mask"])
+    st, sk = oracle_mod.moments(b2["scores"])
+    bud = oracle_mod.allocate(st, sk, Nv, 0.3)
+    cc = oracle_mod.compact(dm2, 0, k2, v2, b2["scores"], bud)
+    for r in range(L * B):
+        l, b = divmod(r, B)
+        first_text = int(cc["offsets"][r]) + int(bud[l, b])
+        assert np.array_equal(cc["k"][first_text:first_text + P], prefix_k[l, b].transpose(1, 0, 2))
+        assert np.array_equal(cc["v"][first_text:first_text + P], prefix_v[l, b].transpose(1, 0, 2))
+
+
 def test_single_row_reduces_to_textbook_softmax(oracle_mod):
     """One head, W = 1: the only elite row sees all visual keys plus its own text key."""
     rng = np.random.default_rng(4)
