@@ -112,6 +112,67 @@ def score(dims: Dims, k: np.ndarray, q_window: np.ndarray, scale: float, alpha: 
     return out
 
 
+def score_groups(dims: Dims, k: np.ndarray, q_window: np.ndarray, scale: float, alpha: float):
+    """Eq. 4-8 with the importance kept apart per KV group -> dict(scores f32 [L,B,Hkv,Nv], elite_mask u64 [L,B,Hq])."""
+    k = _u16(k)
+    q_window = np.ascontiguousarray(_u16(q_window))
+    L, B, Hq, W = dims.n_layers, dims.batch, dims.n_q_heads, dims.window
+    assert k.shape == (L, B, dims.n_kv_heads, dims.n_visual + dims.n_text, dims.head_dim), k.shape
+    assert q_window.shape == (L, B, W, Hq, dims.head_dim), q_window.shape
+    sl, sb, sh, st = full_cache_strides(k)
+    scores = np.empty((L, B, dims.n_kv_heads, dims.n_visual), np.float32)
+    mask = np.empty((L, B, Hq), np.uint64)
+    d = dims.c()
+    rc = lib().oracle_score_groups(C.byref(d), _p(k), C.c_int64(sl), C.c_int64(sb), C.c_int64(sh), C.c_int64(st),
+                                   _p(q_window), C.c_float(scale), C.c_float(alpha), _p(scores), _p(mask))
+    if rc:
+        raise ValueError(f"oracle_score_groups: {rc}")
+    return dict(scores=scores, elite_mask=mask)
+
+
+def allocate_groups(strength: np.ndarray, skewness: np.ndarray, n_visual: int, ratio: float, mode: int = 0):
+    """Eq. 11 over the (layer, KV head) cells of each sequence.  strength/skewness f64 [L,B,Hkv] -> budgets i32."""
+    strength = np.ascontiguousarray(strength, np.float64)
+    skewness = np.ascontiguousarray(skewness, np.float64)
+    L, B, Hkv = strength.shape
+    budgets = np.zeros((L, B, Hkv), np.int32)
+    rc = lib().oracle_allocate_groups(_p(strength), _p(skewness), C.c_int32(L), C.c_int32(B), C.c_int32(Hkv),
+                                      C.c_int32(n_visual), C.c_double(ratio), C.c_int32(mode), _p(budgets))
+    if rc:
+        raise ValueError(f"oracle_allocate_groups: {rc}")
+    return budgets
+
+
+def compact_groups(dims: Dims, slack: int, k: np.ndarray, v: np.ndarray, scores: np.ndarray, budgets: np.ndarray):
+    """Per-KV-group select + gather -> dict(k, v uint16 [rows,1,d], offsets i64 [cells+1], lens i32 [cells], kept_idx)."""
+    k, v = _u16(k), _u16(v)
+    assert k.shape == v.shape and k.strides == v.strides
+    L, B, Hkv = dims.n_layers, dims.batch, dims.n_kv_heads
+    cells = L * B * Hkv
+    scores = np.ascontiguousarray(scores, np.float32).reshape(cells, dims.n_visual)
+    budgets = np.ascontiguousarray(budgets, np.int32).reshape(cells)
+    rows = int(budgets.sum()) + cells * (dims.n_text + slack)
+    k_out = np.zeros((rows, 1, dims.head_dim), np.uint16)
+    v_out = np.zeros_like(k_out)
+    offsets = np.empty(cells + 1, np.int64)
+    lens = np.empty(cells, np.int32)
+    kept = np.empty(max(int(budgets.sum()), 1), np.int32)
+    sl, sb, sh, st = full_cache_strides(k)
+    d = dims.c()
+    rc = lib().oracle_compact_groups(C.byref(d), C.c_int32(slack), _p(k), _p(v), C.c_int64(sl), C.c_int64(sb),
+                                     C.c_int64(sh), C.c_int64(st), _p(scores), _p(budgets), _p(k_out), _p(v_out),
+                                     _p(offsets), _p(lens), _p(kept))
+    if rc:
+        raise ValueError(f"oracle_compact_groups: {rc}")
+    return dict(k=k_out, v=v_out, offsets=offsets, lens=lens, kept_idx=kept[:int(budgets.sum())])
+
+
+def group_decode_dims(dims: Dims) -> Dims:
+    """The per-KV-group cache seen by decode(): every cell is a region with one KV head and G query heads."""
+    return Dims(dims.n_layers * dims.batch * dims.n_kv_heads, 1, dims.n_q_heads // dims.n_kv_heads, 1,
+                dims.head_dim, dims.n_visual, dims.n_text, dims.window)
+
+
 def moments(scores: np.ndarray):
     """Eq. 9-10 on fp32 scores [..., Nv] -> (strength f64 [...], skewness f64 [...])."""
     scores = np.ascontiguousarray(scores, np.float32)

@@ -15,6 +15,9 @@
  *   oracle_select                 Alg. 1 "I[N_v x r]"         pinned (subset enumeration)
  *   oracle_compact                Alg. 1 Concat(K_v[..], K_t) pinned (r = 1 identity, text rows)
  *   oracle_decode                 Section 3.1 token decoding  pinned (masked dense attention, library SDPA)
+ *   oracle_score_groups, oracle_allocate_groups, oracle_compact_groups
+ *                                 Eq. 8-11 and Alg. 1's second loop per KV group (a refinement the paper does not
+ *                                 evaluate)  pinned (mean over groups = the per-layer score, budget sum, library sort)
  *   End-to-end against the authors' implementation: PARITY UNPINNED -- the
  *   paper prints no worked numerical example.
  *
@@ -100,9 +103,35 @@ static uint64_t elite_of_head(const uint16_t *q_last, const uint16_t *k_cand0, i
  *   text keys are not part of K_vtk, Eq. 6); Eq. 8 averages the visual columns
  *   over the elite rows.  The per-layer score is the plain mean over the Hq heads.
  */
+static int score_worker(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, int64_t s_batch,
+                        int64_t s_head, int64_t s_token, const uint16_t *q_window, float scale, float alpha,
+                        float *scores, uint64_t *elite_mask, double *text_mass, float *elite_logits,
+                        float *group_scores);
+
 int oracle_score(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, int64_t s_batch,
                  int64_t s_head, int64_t s_token, const uint16_t *q_window, float scale, float alpha,
                  float *scores, uint64_t *elite_mask, double *text_mass, float *elite_logits) {
+    return score_worker(dm, k, s_layer, s_batch, s_head, s_token, q_window, scale, alpha, scores, elite_mask,
+                        text_mass, elite_logits, NULL);
+}
+
+/*
+ * Eq. 4-8 with the importance kept apart per KV group (the per-KV-head refinement): group g's score of a visual
+ * token is the plain mean of Eq. 8 over the query heads that read KV head g.
+ *   group_scores  fp32 [L, B, Hkv, Nv]  (output), rounded to fp32 once at the end
+ * The mean of the groups' scores over g is the per-layer score of oracle_score (groups have equal size).
+ */
+int oracle_score_groups(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, int64_t s_batch,
+                        int64_t s_head, int64_t s_token, const uint16_t *q_window, float scale, float alpha,
+                        float *group_scores, uint64_t *elite_mask) {
+    return score_worker(dm, k, s_layer, s_batch, s_head, s_token, q_window, scale, alpha, NULL, elite_mask, NULL,
+                        NULL, group_scores);
+}
+
+static int score_worker(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, int64_t s_batch,
+                        int64_t s_head, int64_t s_token, const uint16_t *q_window, float scale, float alpha,
+                        float *scores, uint64_t *elite_mask, double *text_mass, float *elite_logits,
+                        float *group_scores) {
     const int L = dm->n_layers, B = dm->batch, Hq = dm->n_q_heads, Hkv = dm->n_kv_heads;
     const int d = dm->head_dim, Nv = dm->n_visual, Nt = dm->n_text, W = dm->window;
     if (W < 1 || W > 64 || W > Nt || Hq % Hkv != 0 || Nv < 1) return -1;
@@ -113,9 +142,12 @@ int oracle_score(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, in
     for (int l = 0; l < L; ++l) {
         for (int b = 0; b < B; ++b) {
             double *acc = (double *)calloc((size_t)Nv, sizeof(double));   /* sum over heads of I_h */
+            double *acc_g = (double *)calloc((size_t)Nv, sizeof(double)); /* the same over the heads of one KV group */
             double *logit = (double *)malloc((size_t)Nv * sizeof(double));
             double *per_head = (double *)malloc((size_t)Nv * sizeof(double));
-            if (!acc || !logit || !per_head) { status = -2; free(acc); free(logit); free(per_head); continue; }
+            if (!acc || !acc_g || !logit || !per_head) {
+                status = -2; free(acc); free(acc_g); free(logit); free(per_head); continue;
+            }
             const uint16_t *k_lb = k + (int64_t)l * s_layer + (int64_t)b * s_batch;
             const uint16_t *q_lb = q_window + ((int64_t)l * B + b) * (int64_t)W * Hq * d;
             for (int h = 0; h < Hq; ++h) {
@@ -156,11 +188,21 @@ int oracle_score(const oracle_dims_t *dm, const uint16_t *k, int64_t s_layer, in
                 }
                 /* Eq. 8: average pooling over the elite rows */
                 for (int i = 0; i < Nv; ++i) acc[i] += per_head[i] / (double)n_elite;
+                for (int i = 0; i < Nv; ++i) acc_g[i] += per_head[i] / (double)n_elite;
                 if (text_mass) text_mass[((int64_t)l * B + b) * Hq + h] = tmass / (double)n_elite;
+                if (h % G == G - 1) {   /* last head of KV group g: its mean, then start the next group */
+                    if (group_scores) {
+                        float *og = group_scores + (((int64_t)l * B + b) * Hkv + g) * Nv;
+                        for (int i = 0; i < Nv; ++i) og[i] = (float)(acc_g[i] / (double)G);
+                    }
+                    for (int i = 0; i < Nv; ++i) acc_g[i] = 0.0;
+                }
             }
-            float *out = scores + ((int64_t)l * B + b) * Nv;
-            for (int i = 0; i < Nv; ++i) out[i] = (float)(acc[i] / (double)Hq);
-            free(acc); free(logit); free(per_head);
+            if (scores) {
+                float *out = scores + ((int64_t)l * B + b) * Nv;
+                for (int i = 0; i < Nv; ++i) out[i] = (float)(acc[i] / (double)Hq);
+            }
+            free(acc); free(acc_g); free(logit); free(per_head);
         }
     }
     return status;
@@ -346,6 +388,71 @@ int oracle_compact(const oracle_dims_t *dm, int32_t slack, const uint16_t *k, co
         }
     }
     offsets[(int64_t)L * B] = row;
+    return 0;
+}
+
+/*
+ * Eq. 11 per KV group: the cells (layer, KV head) of one sequence take the place of the layers.  Strength and
+ * skewness are normalised by their mean over the L * Hkv cells of the sequence, and T = round-half-up(ratio * Nv *
+ * L * Hkv) rows are split over the cells exactly as oracle_allocate splits a sequence's rows over its layers
+ * (cell order: layer-major, KV head within the layer; ties to the lower cell).
+ *   strength, skewness  f64 [L, B, Hkv];   budgets  i32 [L, B, Hkv] (output)
+ */
+int oracle_allocate_groups(const double *strength, const double *skewness, int32_t n_layers, int32_t batch,
+                           int32_t n_kv_heads, int32_t n_visual, double ratio, int32_t mode, int32_t *budgets) {
+    const int cells = n_layers * n_kv_heads;
+    double *st = (double *)malloc((size_t)cells * sizeof(double));
+    double *sk = (double *)malloc((size_t)cells * sizeof(double));
+    int32_t *bud = (int32_t *)malloc((size_t)cells * sizeof(int32_t));
+    if (!st || !sk || !bud) { free(st); free(sk); free(bud); return -2; }
+    int rc = 0;
+    for (int b = 0; b < batch && !rc; ++b) {
+        for (int l = 0; l < n_layers; ++l)
+            for (int g = 0; g < n_kv_heads; ++g) {
+                const int64_t at = ((int64_t)l * batch + b) * n_kv_heads + g;
+                st[l * n_kv_heads + g] = strength[at];
+                sk[l * n_kv_heads + g] = skewness[at];
+            }
+        rc = oracle_allocate(st, sk, cells, 1, n_visual, ratio, mode, bud);   /* the cells as the layers of one sequence */
+        for (int l = 0; l < n_layers; ++l)
+            for (int g = 0; g < n_kv_heads; ++g)
+                budgets[((int64_t)l * batch + b) * n_kv_heads + g] = bud[l * n_kv_heads + g];
+    }
+    free(st); free(sk); free(bud);
+    return rc;
+}
+
+/*
+ * Alg. 1's second loop per KV group: cell (l, b, g) keeps its own budgets[l, b, g] visual tokens of largest
+ * group score and all text tokens; rows are single-head rows of d elements.  Cell index c = (l*B + b)*Hkv + g,
+ * first row offsets[c] = sum over c' < c of (budget[c'] + Nt + slack).
+ *   k_out, v_out  bf16 [rows, d];  offsets i64 [L*B*Hkv + 1];  lens i32 [L*B*Hkv];  kept_idx packed per cell
+ */
+int oracle_compact_groups(const oracle_dims_t *dm, int32_t slack, const uint16_t *k, const uint16_t *v,
+                          int64_t s_layer, int64_t s_batch, int64_t s_head, int64_t s_token,
+                          const float *group_scores, const int32_t *budgets, uint16_t *k_out, uint16_t *v_out,
+                          int64_t *offsets, int32_t *lens, int32_t *kept_idx) {
+    const int L = dm->n_layers, B = dm->batch, Hkv = dm->n_kv_heads, d = dm->head_dim;
+    const int Nv = dm->n_visual, Nt = dm->n_text;
+    int64_t row = 0, kept_pos = 0;
+    for (int64_t c = 0; c < (int64_t)L * B * Hkv; ++c) {
+        const int g = (int)(c % Hkv), b = (int)(c / Hkv % B), l = (int)(c / Hkv / B);
+        const int32_t n = budgets[c];
+        offsets[c] = row;
+        lens[c] = n + Nt;
+        int32_t *kept = kept_idx + kept_pos;
+        int rc = oracle_select(group_scores + c * Nv, Nv, n, kept);
+        if (rc) return rc;
+        for (int j = 0; j < n + Nt; ++j) {
+            const int64_t tok = (j < n) ? kept[j] : (int64_t)Nv + (j - n);
+            const int64_t src = (int64_t)l * s_layer + (int64_t)b * s_batch + (int64_t)g * s_head + tok * s_token;
+            memcpy(k_out + (row + j) * d, k + src, (size_t)d * sizeof(uint16_t));
+            memcpy(v_out + (row + j) * d, v + src, (size_t)d * sizeof(uint16_t));
+        }
+        row += n + Nt + slack;
+        kept_pos += n;
+    }
+    offsets[(int64_t)L * B * Hkv] = row;
     return 0;
 }
 

@@ -416,6 +416,95 @@ def test_select_equal_scores_and_planted_subset(oracle_mod):
 
 
 # ----------------------------------------------------------------------------------------------
+# per-KV-group budgets (Eq. 8-11 and the second loop of Algorithm 1 applied to every KV head on its own)
+# ----------------------------------------------------------------------------------------------
+def test_group_scores_average_to_the_layer_score_and_match_the_matrix_form(oracle_mod):
+    rng = np.random.default_rng(41)
+    L, B, Hq, Hkv, d, Nv, Nt, W = 2, 2, 6, 3, 16, 33, 9, 5
+    k, _, qw = rand_case(rng, L, B, Hq, Hkv, d, Nv, Nt, W)
+    dm = oracle_mod.Dims(L, B, Hq, Hkv, d, Nv, Nt, W)
+    scale = 1 / math.sqrt(d)
+    whole = oracle_mod.score(dm, k, qw, scale, 0.7)
+    grp = oracle_mod.score_groups(dm, k, qw, scale, 0.7)
+    assert np.array_equal(whole["elite_mask"], grp["elite_mask"])
+    # groups have equal size: the mean over the groups is the mean over all heads (one fp32 rounding apart)
+    assert np.allclose(grp["scores"].astype(np.float64).mean(axis=2), whole["scores"], rtol=3e-7, atol=0)
+    # and each group's score is the library-softmax matrix form averaged over that group's heads only
+    kf, qf = bf16_val(k), bf16_val(qw)
+    G = Hq // Hkv
+    for l, b, g in itertools.product(range(L), range(B), range(Hkv)):
+        acc = np.zeros(Nv)
+        for h in range(g * G, (g + 1) * G):
+            iv, _ = literal_importance(kf[l, b, g], qf[l, b, :, h, :], int(grp["elite_mask"][l, b, h]), Nv, Nt, W, scale)
+            acc += iv
+        assert np.allclose(grp["scores"][l, b, g], acc / G, rtol=2e-7, atol=0)
+    # heads of different groups do not leak into each other: changing group 1's keys leaves group 0's score alone
+    k2 = k.copy()
+    k2[:, :, 1] = bf16_bits(rng.standard_normal(k2[:, :, 1].shape))
+    grp2 = oracle_mod.score_groups(dm, k2, qw, scale, 0.7)
+    assert np.array_equal(grp2["scores"][:, :, 0], grp["scores"][:, :, 0])
+    assert not np.array_equal(grp2["scores"][:, :, 1], grp["scores"][:, :, 1])
+
+
+def test_group_budgets_sum_cap_and_reduce_to_the_layer_rule(oracle_mod):
+    rng = np.random.default_rng(42)
+    L, B, Hkv, Nv = 5, 3, 4, 50
+    for ratio in (0.0, 0.1, 0.37, 0.9, 1.0):
+        st = rng.uniform(0.1, 1.0, (L, B, Hkv))
+        sk = rng.uniform(-1.0, 6.0, (L, B, Hkv))
+        bud = oracle_mod.allocate_groups(st, sk, Nv, ratio)
+        assert bud.shape == (L, B, Hkv) and bud.min() >= 0 and bud.max() <= Nv
+        T = oracle_mod.total_kept(Nv, L * Hkv, ratio)
+        assert (bud.sum(axis=(0, 2)) == T).all()
+        # a sequence's cells are apportioned exactly like the layers of a sequence with L * Hkv layers
+        for b in range(B):
+            flat = oracle_mod.allocate(st[:, b].reshape(L * Hkv, 1), sk[:, b].reshape(L * Hkv, 1), Nv, ratio)
+            assert np.array_equal(bud[:, b].reshape(-1), flat[:, 0])
+    # one KV head: the per-layer rule itself
+    st, sk = rng.uniform(0.1, 1.0, (L, B, 1)), rng.uniform(0.0, 3.0, (L, B, 1))
+    assert np.array_equal(oracle_mod.allocate_groups(st, sk, Nv, 0.3)[:, :, 0], oracle_mod.allocate(st[:, :, 0], sk[:, :, 0], Nv, 0.3))
+    # equal cells: a uniform split with the spare rows on the lowest cells
+    bud = oracle_mod.allocate_groups(np.ones((3, 1, 2)), np.ones((3, 1, 2)), 10, 0.45)   # T = 27 over 6 cells
+    assert bud.reshape(-1).tolist() == [5, 5, 5, 4, 4, 4]
+
+
+def test_group_compaction_keeps_each_heads_own_tokens_and_all_text(oracle_mod):
+    rng = np.random.default_rng(43)
+    L, B, Hq, Hkv, d, Nv, Nt, W = 2, 2, 4, 2, 16, 40, 6, 4
+    k, v, qw = rand_case(rng, L, B, Hq, Hkv, d, Nv, Nt, W)
+    dm = oracle_mod.Dims(L, B, Hq, Hkv, d, Nv, Nt, W)
+    sc = oracle_mod.score_groups(dm, k, qw, 0.25, 0.9)["scores"]
+    st, sk = oracle_mod.moments(sc)
+    bud = oracle_mod.allocate_groups(st, sk, Nv, 0.25)
+    slack = 2
+    cc = oracle_mod.compact_groups(dm, slack, k, v, sc, bud)
+    pos = 0
+    for c in range(L * B * Hkv):
+        l, b, g = c // Hkv // B, c // Hkv % B, c % Hkv
+        n = int(bud[l, b, g])
+        want = np.sort(np.lexsort((np.arange(Nv), -sc[l, b, g]))[:n])     # library sort: top n, ties to the lower index
+        assert cc["kept_idx"][pos:pos + n].tolist() == want.tolist()
+        a = int(cc["offsets"][c])
+        assert int(cc["lens"][c]) == n + Nt and int(cc["offsets"][c + 1]) - a == n + Nt + slack
+        assert np.array_equal(cc["k"][a:a + n, 0], k[l, b, g, want])
+        assert np.array_equal(cc["v"][a:a + n, 0], v[l, b, g, want])
+        assert np.array_equal(cc["k"][a + n:a + n + Nt, 0], k[l, b, g, Nv:])
+        assert np.array_equal(cc["v"][a + n:a + n + Nt, 0], v[l, b, g, Nv:])
+        pos += n
+    # full retention: decode over the per-group cache equals decode over the full cache
+    bud1 = np.full((L, B, Hkv), Nv, np.int32)
+    c1 = oracle_mod.compact_groups(dm, 0, k, v, sc, bud1)
+    q = bf16_bits(rng.standard_normal((L, B, Hq, d)))
+    got = oracle_mod.decode(oracle_mod.group_decode_dims(dm), c1["k"], c1["v"], c1["offsets"], c1["lens"],
+                            q.reshape(L * B * Hkv, 1, Hq // Hkv, d), 0.25).reshape(L, B, Hq, d)
+    N = Nv + Nt
+    kf = np.ascontiguousarray(k.transpose(0, 1, 3, 2, 4)).reshape(L * B * N, Hkv, d)
+    vf = np.ascontiguousarray(v.transpose(0, 1, 3, 2, 4)).reshape(L * B * N, Hkv, d)
+    want = oracle_mod.decode(dm, kf, vf, (np.arange(L * B + 1) * N).astype(np.int64), np.full(L * B, N, np.int32), q, 0.25)
+    assert np.allclose(got, want, rtol=1e-6, atol=1e-7)
+
+
+# ----------------------------------------------------------------------------------------------
 # compaction and decode
 # ----------------------------------------------------------------------------------------------
 def small_pipeline(oracle_mod, ratio, slack=0, seed=14):
