@@ -49,7 +49,7 @@
 extern "C" {
 #endif
 
-#define AIRCACHE_VERSION 100
+#define AIRCACHE_VERSION 101
 
 #define AIRCACHE_OK 0
 #define AIRCACHE_ERR_INVALID_ARG (-1)          /* NULL pointer, negative size, ratio outside [0,1], ...        */
@@ -67,7 +67,7 @@ extern "C" {
 /* Problem shape, uniform over the batch. */
 typedef struct {
     int32_t n_layers;    /* L >= 1                                                                   */
-    int32_t batch;       /* B >= 1; L * B <= 1792                                                    */
+    int32_t batch;       /* B >= 1; L * B <= 1792 (L * B * Hkv <= 1792 with per_kv_head)             */
     int32_t n_q_heads;   /* Hq, a multiple of n_kv_heads with Hq / Hkv <= 16                         */
     int32_t n_kv_heads;  /* Hkv in {1, 2, 4, 8}                                                      */
     int32_t head_dim;    /* d in {64, 128}                                                           */
@@ -76,7 +76,26 @@ typedef struct {
     int32_t window;      /* W: the last W text tokens are the candidates of Eq. 5; 1 <= W <= min(64, Nt) */
     int32_t slack;       /* rows left free after each region for tokens appended while decoding, >= 0 */
     float scale;         /* softmax scale of Eq. 4 and Eq. 7, normally 1 / sqrt(head_dim)            */
+    int32_t per_kv_head; /* 0: one budget and one kept set per (layer, sequence), shared by all KV heads
+                            (the paper's method).  1: Eq. 8-11 and the top-k of Algorithm 1 applied to
+                            every KV head on its own - see "Per-KV-head mode" below                  */
 } aircache_shape_t;
+
+/*
+ * Per-KV-head mode (per_kv_head = 1), a refinement the paper does not evaluate.
+ * The unit of compression is the cell (layer l, sequence b, KV head g), index
+ * c = (l * B + b) * Hkv + g, instead of the region (l, b):
+ *   scores    fp32 [L, B, Hkv, Nv]: Eq. 8 averaged over the query heads of group g only;
+ *   budgets, strength, skewness  [L, B, Hkv]: Eq. 9-10 per cell; Eq. 11 normalises over the
+ *             L * Hkv cells of a sequence, which share T = floor(ratio * Nv * L * Hkv + 0.5)
+ *             rows (aircache_kept_per_sequence), ties to the lower cell;
+ *   ragged cache: rows are single-head rows, k and v bf16 [total_rows, 1, d]; offsets
+ *             [L*B*Hkv + 1] and lens [L*B*Hkv] are per cell; cell c keeps its own tokens;
+ *   kept_idx  cell c's ascending list at offsets[c] - c * (Nt + slack);
+ *   decode    query head h attends to the cell of its KV head; q and out stay [L, B, Hq, d];
+ *   append    k_new, v_new stay [L, B, Hkv, d]: one row per cell.
+ * Everything else (elite_mask, window queries, the full cache view) is unchanged.
+ */
 
 /*
  * Full (uncompressed) cache of the prefill: logical bf16 [L, B, Hkv, Nv+Nt, d]
@@ -184,8 +203,8 @@ int aircache_score_layers(const aircache_shape_t *shape, const aircache_full_t *
  * every layer capped at Nv (excess re-shared), floors first, the remaining rows
  * one each to the largest fractional parts, ties to the lower layer.
  *   mode      0: Eq. 11   1: strength only   2: skewness only   3: uniform
- *   budgets   i32 [L, B]  output n_{l,b}
- *   strength, skewness  f64 [L, B]  outputs; either may be NULL
+ *   budgets   i32 [L, B]  output n_{l,b}                       ([L, B, Hkv] in per-KV-head mode,
+ *   strength, skewness  f64 [L, B]  outputs; either may be NULL  as are these)
  *   layout    offsets and lens are written (offsets[r+1] - offsets[r] = n_r + Nt + slack,
  *             lens[r] = n_r + Nt); k and v are not touched
  */
@@ -333,7 +352,7 @@ int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes);
  *   d_scores     DEVICE fp32 [L, B, Nv];  d_budgets DEVICE i32 [L, B]
  *   d_cache      DEVICE ragged cache (k, v, offsets, lens, total_rows)
  *   d_out        DEVICE fp32 [n_steps, L, B, Hq, d];  h_out HOST, same size (output)
- *   h_budgets    HOST i32 [L, B] (output)
+ *   h_budgets    HOST i32 [L, B] (output; [L, B, Hkv] in per-KV-head mode, like d_budgets)
  */
 int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t *h_full, int64_t full_elems,
                            void *d_full_k, void *d_full_v, const void *h_q_window, void *d_q_window,

@@ -36,7 +36,8 @@ class AirCacheError(RuntimeError):
 
 class Shape(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_visual",
-                                           "n_text", "window", "slack")] + [("scale", C.c_float)]
+                                           "n_text", "window", "slack")] + [("scale", C.c_float),
+                                                                            ("per_kv_head", C.c_int32)]
 
 
 class Full(C.Structure):
@@ -129,10 +130,12 @@ def _check(fn: str, rc: int) -> None:
         raise AirCacheError(fn, rc)
 
 
-def shape(n_layers, batch, n_q_heads, n_kv_heads, head_dim, n_visual, n_text, window, slack=0, scale=None) -> Shape:
+def shape(n_layers, batch, n_q_heads, n_kv_heads, head_dim, n_visual, n_text, window, slack=0, scale=None,
+          per_kv_head=0) -> Shape:
     if scale is None:
         scale = 1.0 / math.sqrt(head_dim)   # rounded to fp32 by ctypes
-    return Shape(n_layers, batch, n_q_heads, n_kv_heads, head_dim, n_visual, n_text, window, slack, scale)
+    return Shape(n_layers, batch, n_q_heads, n_kv_heads, head_dim, n_visual, n_text, window, slack, scale,
+                 int(per_kv_head))
 
 
 def full_view(k: torch.Tensor, v: torch.Tensor) -> Full:

@@ -26,7 +26,8 @@ int check_shape(const aircache_shape_t *s) {
     if (s->n_q_heads / s->n_kv_heads > kMaxGroup) return AIRCACHE_ERR_UNSUPPORTED;
     if (s->window > kMaxWindow) return AIRCACHE_ERR_UNSUPPORTED;
     if (s->n_visual < 3) return AIRCACHE_ERR_UNSUPPORTED;
-    if ((int64_t)s->n_layers * s->batch > kMaxRegions) return AIRCACHE_ERR_UNSUPPORTED;
+    if (s->per_kv_head != 0 && s->per_kv_head != 1) return AIRCACHE_ERR_INVALID_ARG;
+    if (n_cells(s) > kMaxRegions) return AIRCACHE_ERR_UNSUPPORTED;
     if ((int64_t)s->n_visual + s->n_text + s->slack > (1 << 24)) return AIRCACHE_ERR_UNSUPPORTED;
     return AIRCACHE_OK;
 }
@@ -44,7 +45,7 @@ int check_full(const aircache_shape_t *s, const aircache_full_t *f) {
 }
 
 int64_t kept_per_sequence(const aircache_shape_t *s, double ratio) {
-    int64_t cells = (int64_t)s->n_visual * (int64_t)s->n_layers;
+    int64_t cells = (int64_t)s->n_visual * (int64_t)s->n_layers * cells_of(s);
     return (int64_t)floor(ratio * (double)cells + 0.5);
 }
 
@@ -70,9 +71,9 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.chunk_stats = take(groups * chunks * cap * 8);
     w.row_final = take(groups * cap * 8);
     w.group_ticket = take(groups * 4);
-    w.mom_strength = take(LB * 8);
-    w.mom_skew = take(LB * 8);
-    w.kept = take(LB * s->n_visual * 4);
+    w.mom_strength = take(n_cells(s) * 8);
+    w.mom_skew = take(n_cells(s) * 8);
+    w.kept = take(n_cells(s) * s->n_visual * 4);
     w.partials = take((int64_t)2 * kMaxDecodeCtas * partial_slot_floats(s->n_q_heads, s->head_dim) * 4);
     w.total = off;
     return w;
@@ -160,7 +161,7 @@ int64_t aircache_kept_per_sequence(const aircache_shape_t *shape, double ratio) 
 int64_t aircache_total_rows(const aircache_shape_t *shape, double ratio) {
     int64_t t = aircache_kept_per_sequence(shape, ratio);
     if (t < 0) return t;
-    return (int64_t)shape->batch * (t + (int64_t)shape->n_layers * ((int64_t)shape->n_text + shape->slack));
+    return (int64_t)shape->batch * (t + (int64_t)shape->n_layers * cells_of(shape) * ((int64_t)shape->n_text + shape->slack));
 }
 
 int64_t aircache_workspace_bytes(const aircache_shape_t *shape) {
@@ -400,7 +401,7 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
                                               side.stream));
         }
     }
-    AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_budgets, d_budgets, LB * 4, cudaMemcpyDeviceToHost, st));
+    AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_budgets, d_budgets, n_cells(shape) * 4, cudaMemcpyDeviceToHost, st));
     if (n_steps > 0) AIRCACHE_CUDA_TRY(cudaStreamSynchronize(side.stream));
     AIRCACHE_CUDA_TRY(cudaStreamSynchronize(st));
     return AIRCACHE_OK;

@@ -26,7 +26,7 @@ struct BudgetParams {
     int64_t *offsets;        // [L*B+1]
     int32_t *lens;           // [L*B]
     uint32_t *ticket;        // zero between calls
-    int L, B, Nv, Nt, slack, mode;
+    int L, B, Hc, Nv, Nt, slack, mode;   // Hc: cells per (layer, sequence) - the KV heads in per-KV-head mode, else 1
     long long total_kept;    // T per sequence
     long long first_row;     // rows of the shared buffers in front of this cache's first region
 };
@@ -48,17 +48,21 @@ __device__ __forceinline__ double warp_bcast(double v, int src) {
     return __shfl_sync(0xffffffffu, v, src);
 }
 
-// Eq. 11 and the integer budgets of sequence b, by one warp.  st/sk/w/share are [L*B] arrays in shared
-// memory, element (l, b) at l*B + b; act flags layers that still take part in the proportional split.
+// Eq. 11 and the integer budgets of sequence b, by one warp.  st/sk/w/share are arrays over all cells in shared
+// memory; the sequence's cells - its layers, or its (layer, KV head) pairs in per-KV-head mode, layer-major -
+// are numbered l = 0 .. L*Hc - 1 here and sit at AT(l); act flags cells that still take part in the
+// proportional split.
 __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st, const double *sk, double *w,
                                   double *share, unsigned char *act, int *bud) {
-    const int L = p.L, B = p.B, lane = threadIdx.x & 31;
+    const int L = p.L * p.Hc, lane = threadIdx.x & 31;
+    const int B = p.B, Hc = p.Hc;
+#define AT(l) ((((l) / Hc) * B + b) * Hc + (l) % Hc)
     // across-layer means: one lane, layer order (this fixes the rounding of the sums)
     double mean_t = 0.0, mean_k = 0.0;
     if (lane == 0) {
         for (int l = 0; l < L; ++l) {
-            mean_t = __dadd_rn(mean_t, st[l * B + b]);
-            const double s = sk[l * B + b];
+            mean_t = __dadd_rn(mean_t, st[AT(l)]);
+            const double s = sk[AT(l)];
             mean_k = __dadd_rn(mean_k, s > 0.0 ? s : 0.0);
         }
         mean_t = __ddiv_rn(mean_t, (double)L);
@@ -67,8 +71,8 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     mean_t = warp_bcast(mean_t, 0);
     mean_k = warp_bcast(mean_k, 0);
     for (int l = lane; l < L; l += 32) {
-        const double t = st[l * B + b];
-        double s = sk[l * B + b];
+        const double t = st[AT(l)];
+        double s = sk[AT(l)];
         if (s < 0.0) s = 0.0;
         const double nt = mean_t > 0.0 ? __ddiv_rn(t, mean_t) : 1.0;
         const double nk = mean_k > 0.0 ? __ddiv_rn(s, mean_k) : 1.0;
@@ -77,8 +81,8 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
         else if (p.mode == 1) ww = nt;
         else if (p.mode == 2) ww = nk;
         else ww = 1.0;
-        w[l * B + b] = ww;
-        act[l * B + b] = 1;
+        w[AT(l)] = ww;
+        act[AT(l)] = 1;
     }
     __syncwarp();
     long long R = p.total_kept;
@@ -88,20 +92,20 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
         int n_active = 0;
         if (lane == 0) {
             for (int l = 0; l < L; ++l)
-                if (act[l * B + b]) { wsum = __dadd_rn(wsum, w[l * B + b]); ++n_active; }
+                if (act[AT(l)]) { wsum = __dadd_rn(wsum, w[AT(l)]); ++n_active; }
         }
         wsum = warp_bcast(wsum, 0);
         n_active = __shfl_sync(0xffffffffu, n_active, 0);
         if (n_active == 0) break;
         int moved = 0;
         for (int l = lane; l < L; l += 32) {
-            if (!act[l * B + b]) continue;
-            const double sh = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, w[l * B + b]), wsum)
+            if (!act[AT(l)]) continue;
+            const double sh = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, w[AT(l)]), wsum)
                                          : __ddiv_rn((double)R, (double)n_active);
-            share[l * B + b] = sh;
+            share[AT(l)] = sh;
             if (sh >= (double)p.Nv) {
-                bud[l * B + b] = p.Nv;
-                act[l * B + b] = 0;
+                bud[AT(l)] = p.Nv;
+                act[AT(l)] = 0;
                 ++moved;
             }
         }
@@ -114,12 +118,12 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     // floors, then the largest fractional parts (ties to the lower layer) take one more row each
     int given = 0;
     for (int l = lane; l < L; l += 32) {
-        if (!act[l * B + b]) continue;
-        const double sh = share[l * B + b];
+        if (!act[AT(l)]) continue;
+        const double sh = share[AT(l)];
         const int f = (int)floor(sh);
-        bud[l * B + b] = f;
+        bud[AT(l)] = f;
         given += f;
-        share[l * B + b] = __dsub_rn(sh, (double)f);
+        share[AT(l)] = __dsub_rn(sh, (double)f);
     }
     long long given_all = given;
 #pragma unroll
@@ -129,27 +133,28 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     // a layer gets the extra row iff fewer than `left` active layers precede it in the order
     // (fraction descending, layer ascending): the same set the one-at-a-time selection picks
     for (int l = lane; l < L; l += 32) {
-        if (!act[l * B + b]) continue;
-        const double fr = share[l * B + b];
+        if (!act[AT(l)]) continue;
+        const double fr = share[AT(l)];
         long long rank = 0;
         for (int l2 = 0; l2 < L; ++l2) {
-            if (!act[l2 * B + b]) continue;
-            const double f2 = share[l2 * B + b];
+            if (!act[AT(l2)]) continue;
+            const double f2 = share[AT(l2)];
             rank += (f2 > fr) || (f2 == fr && l2 < l);
         }
-        if (rank < left) bud[l * B + b] += 1;
+        if (rank < left) bud[AT(l)] += 1;
     }
     __syncwarp();
 }
+#undef AT
 
 __global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ double s_part[kThreads / 32];
     __shared__ int s_is_last;
     const int tid = threadIdx.x;
-    const int LB = p.L * p.B;
+    const int LB = p.L * p.B * p.Hc;   // cells
 
-    // ---------------- Eq. 9 and Eq. 10 of region blockIdx.x ----------------
+    // ---------------- Eq. 9 and Eq. 10 of cell blockIdx.x ----------------
     {
         const float *x = p.scores + (int64_t)blockIdx.x * p.Nv;
         const double n = (double)p.Nv;
@@ -264,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
 int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, int32_t mode, int32_t *budgets,
                   double *strength, double *skewness, aircache_ragged_t *layout, void *ws, cudaStream_t st) {
     const WsLayout w = ws_layout(s);
-    const int LB = s->n_layers * s->batch;
+    const int LB = (int)n_cells(s);
     BudgetParams p;
     p.scores = scores;
     p.strength = strength ? strength : ws_ptr<double>(ws, w.mom_strength);
@@ -273,7 +278,7 @@ int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, 
     p.offsets = layout->offsets;
     p.lens = layout->lens;
     p.ticket = ws_ptr<uint32_t>(ws, w.status) + 2;   // second word pair of the status block
-    p.L = s->n_layers; p.B = s->batch; p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack; p.mode = mode;
+    p.L = s->n_layers; p.B = s->batch; p.Hc = cells_of(s); p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack; p.mode = mode;
     p.total_kept = kept_per_sequence(s, ratio);
     p.first_row = layout->first_row;
     const size_t smem = (size_t)LB * (4 * 8 + 4 + 1) + 16;

@@ -57,6 +57,12 @@ int64_t kept_per_sequence(const aircache_shape_t *s, double ratio);
 
 inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
+// Cells per (layer, sequence): the units that get a budget, a kept set and a stretch of the ragged cache of their
+// own - the KV heads in per-KV-head mode, else the region as a whole.  KV heads stored in one row of the cache.
+inline int cells_of(const aircache_shape_t *s) { return s->per_kv_head ? s->n_kv_heads : 1; }
+inline int row_heads_of(const aircache_shape_t *s) { return s->per_kv_head ? 1 : s->n_kv_heads; }
+inline int64_t n_cells(const aircache_shape_t *s) { return (int64_t)s->n_layers * s->batch * cells_of(s); }
+
 // Floats of one split-K partial slot of the decode kernel: [Hq, d] accumulator, Hq maxima, Hq sums, padded so
 // that every slot starts on a 16-byte boundary.
 __host__ __device__ inline int64_t partial_slot_floats(int n_q_heads, int head_dim) {
@@ -99,9 +105,9 @@ struct WsLayout {
     int64_t chunk_stats;  // f32x2[L*B*Hkv][chunks][cap]  (max, sum) over one chunk of visual keys
     int64_t row_final;    // f32x2[L*B*Hkv][cap]       (max, weight / normaliser) after all chunks
     int64_t group_ticket; // u32  [L*B*Hkv]            chunks of the group done so far
-    int64_t mom_strength; // f64  [L*B]
-    int64_t mom_skew;     // f64  [L*B]
-    int64_t kept;         // i32  [L*B*Nv]             kept-token lists when the caller passes none
+    int64_t mom_strength; // f64  [cells]
+    int64_t mom_skew;     // f64  [cells]
+    int64_t kept;         // i32  [cells*Nv]           kept-token lists when the caller passes none
     int64_t partials;     // f32  [2*kMaxDecodeCtas][Hq*(d+2)]
     int64_t total;
 };

@@ -170,6 +170,7 @@ struct GatherParams {
     int64_t rows_cap;  // rows covered by the launch
     int64_t first_row; // rows of the shared buffers in front of this cache's first region
     int L, B, Hkv, d, Nv, Nt, slack;
+    int Hc;   // cells per (layer, sequence): 1, or the KV heads in per-KV-head mode (a row then holds one head)
 };
 
 constexpr int kGatherThreads = 256;
@@ -185,9 +186,16 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kGatherThreads + threadIdx.x) >> 5;
     const int64_t row_step = (int64_t)gridDim.x * (kGatherThreads / 32) * kGatherRowsPerWarp;
-    const int n_regions = p.L * p.B;
+    const int n_regions = p.L * p.B * p.Hc;       // cells
+    const int row_heads = p.Hc > 1 ? 1 : p.Hkv;   // KV heads in one row of the ragged cache
     const int vec_per_head = p.d / 8;             // 16-byte vectors per head slice
-    const int vec_per_row = p.Hkv * vec_per_head;
+    const int vec_per_row = row_heads * vec_per_head;
+    // source offset of token `tok` of cell r (its first head's slice)
+    auto src_of = [&](int r, int tok) {
+        const int lb = r / p.Hc, g0 = r - lb * p.Hc;
+        const int l = lb / p.B, b = lb - l * p.B;
+        return (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g0 * p.s_head + (int64_t)tok * p.s_token;
+    };
 
     auto copy_rows = [&](const int64_t (&src_off)[kGatherRowsPerWarp], const int64_t (&dst_row)[kGatherRowsPerWarp]) {
         for (int v0 = lane; v0 < vec_per_row; v0 += 32) {
@@ -203,7 +211,7 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
 #pragma unroll
             for (int i = 0; i < kGatherRowsPerWarp; ++i) {
                 if (dst_row[i] < 0) continue;
-                const int64_t dof = (dst_row[i] * p.Hkv + g) * p.d + c * 8;
+                const int64_t dof = (dst_row[i] * row_heads + g) * p.d + c * 8;
                 *reinterpret_cast<uint4 *>(p.k_out + dof) = kk[i];
                 *reinterpret_cast<uint4 *>(p.v_out + dof) = vv[i];
             }
@@ -221,8 +229,7 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
             src_off[i] = 0;
             if (idx >= n_text_rows) continue;
             const int r = idx / p.Nt, j = idx - r * p.Nt;
-            const int l = r / p.B, b = r - l * p.B;
-            src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)(p.Nv + j) * p.s_token;
+            src_off[i] = src_of(r, p.Nv + j);
             dst_row[i] = p.offsets[r] + p.budgets[r] + j;
         }
         copy_rows(src_off, dst_row);
@@ -249,8 +256,7 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
             const int r = lo;
             const int64_t base = p.offsets[r];
             const int j = (int)(idx - (base - p.first_row - (int64_t)r * per));
-            const int l = r / p.B, b = r - l * p.B;
-            src_off[i] = (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)p.kept[idx] * p.s_token;
+            src_off[i] = src_of(r, p.kept[idx]);
             dst_row[i] = base + j;
         }
         copy_rows(src_off, dst_row);
@@ -276,7 +282,7 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
                    const int32_t *budgets, double ratio, aircache_ragged_t *out, int32_t *kept_idx, void *ws,
                    cudaStream_t st) {
     const WsLayout w = ws_layout(s);
-    const int LB = s->n_layers * s->batch;
+    const int LB = (int)n_cells(s);
     int32_t *kept = kept_idx ? kept_idx : ws_ptr<int32_t>(ws, w.kept);
     if (s->n_visual <= kSelSmemKeys) {
         const size_t smem = (size_t)s->n_visual * 4;
@@ -296,7 +302,8 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     p.k_out = (uint16_t *)out->k; p.v_out = (uint16_t *)out->v;
     p.offsets = out->offsets; p.lens = out->lens; p.budgets = budgets; p.kept = kept;
     p.first_row = out->first_row;
-    p.rows_cap = (int64_t)s->batch * (kept_per_sequence(s, ratio) + (int64_t)s->n_layers * (s->n_text + s->slack));
+    p.rows_cap = (int64_t)s->batch * kept_per_sequence(s, ratio) + (int64_t)LB * (s->n_text + s->slack);
+    p.Hc = cells_of(s);
     p.L = s->n_layers; p.B = s->batch; p.Hkv = s->n_kv_heads; p.d = s->head_dim;
     p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack;
     const int64_t rows_per_block = (kGatherThreads / 32) * kGatherRowsPerWarp;
@@ -326,9 +333,9 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
 int launch_append(const aircache_shape_t *s, aircache_ragged_t *c, const void *k_new, const void *v_new,
                   int32_t appended, cudaStream_t st) {
     (void)appended;
-    append_kernel<<<s->n_layers * s->batch, 64, 0, st>>>((uint16_t *)c->k, (uint16_t *)c->v, c->offsets, c->lens,
-                                                         (const uint16_t *)k_new, (const uint16_t *)v_new,
-                                                         s->n_kv_heads * s->head_dim);
+    append_kernel<<<(unsigned)n_cells(s), 64, 0, st>>>((uint16_t *)c->k, (uint16_t *)c->v, c->offsets, c->lens,
+                                                       (const uint16_t *)k_new, (const uint16_t *)v_new,
+                                                       row_heads_of(s) * s->head_dim);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
 }

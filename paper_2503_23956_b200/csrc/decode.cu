@@ -1218,6 +1218,23 @@ int launch_decode_d(const aircache_shape_t *s, const aircache_ragged_t *c, Decod
     }
 }
 
+// In per-KV-head mode every cell (layer, sequence, KV head) is a region of its own with one KV head and the G query
+// heads that read it: q and out [L, B, Hq, d] are [cells, G, d] as they stand, the new token's rows [cells, 1, d].
+// The kernel sees that shape; the workspace carve-up stays the caller's.
+const aircache_shape_t *decode_view(const aircache_shape_t *s, DecodeParams &p, aircache_shape_t *view) {
+    if (!s->per_kv_head) return s;
+    *view = *s;
+    view->n_layers = (int32_t)n_cells(s);
+    view->batch = 1;
+    view->n_q_heads = s->n_q_heads / s->n_kv_heads;
+    view->n_kv_heads = 1;
+    view->per_kv_head = 0;
+    p.n_regions = view->n_layers;
+    p.Hq = view->n_q_heads;
+    p.kv_heads = 1;
+    return view;
+}
+
 }  // namespace
 
 int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const void *q, const void *k_new,
@@ -1244,6 +1261,8 @@ int launch_decode(const aircache_shape_t *s, const aircache_ragged_t *c, const v
     p.G = s->n_q_heads / s->n_kv_heads;
     p.sl2 = s->scale * kLog2e;
     p.hs = 1;
+    aircache_shape_t view;
+    s = decode_view(s, p, &view);
     return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
 }
 
@@ -1302,6 +1321,8 @@ int launch_decode_static(const aircache_shape_t *s, const aircache_ragged_t *c, 
     p.G = s->n_q_heads / s->n_kv_heads;
     p.sl2 = s->scale * kLog2e;
     p.hs = 1;
+    aircache_shape_t view;
+    s = decode_view(s, p, &view);
     return s->head_dim == 64 ? launch_decode_d<64>(s, c, p, st) : launch_decode_d<128>(s, c, p, st);
 }
 

@@ -42,6 +42,7 @@ struct ScoreParams {
     uint32_t *group_ticket;
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
     int lb0, n_lb;   // the launch covers regions lb0 .. lb0 + n_lb - 1 (a range of layers)
+    int per_head;    // scores are kept apart per KV group: [L,B,Hkv,Nv], Eq. 8 averaged over the group's heads only
     int cap, chunks, chunk_keys;
     float scale, sl2, ln_alpha;
     int keep_all;
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         if (!((mask >> w) & 1)) continue;
         const int r = s_first_row[hl] + __popcll(mask & (((uint64_t)1 << w) - 1));
         info[r] = (hl << 8) | w;
-        coef[r] = 1.0f / ((float)__popcll(mask) * (float)p.Hq);
+        coef[r] = 1.0f / ((float)__popcll(mask) * (float)(p.per_head ? p.G : p.Hq));
         // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.  The query row goes to registers
         // once, the keys come from shared memory.
         uint4 qr[D / 8];
@@ -412,17 +413,21 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
                 }
             }
         }
-    }
-    float *out = p.scores + (int64_t)lb * p.Nv;
+        if (p.per_head || g == p.Hkv - 1) {
+            // the key's score is complete: of this KV group alone, or summed over all of them
+            float *out = p.scores + (p.per_head ? (int64_t)grp : (int64_t)lb) * p.Nv;
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
+            for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            float v = imp[mt][j];
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            const int key = kbase + mt * 16 + gid + 8 * j;
-            if (t == 0 && key < p.Nv) out[key] = v;
+                for (int j = 0; j < 2; ++j) {
+                    float v = imp[mt][j];
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    const int key = kbase + mt * 16 + gid + 8 * j;
+                    if (t == 0 && key < p.Nv) out[key] = v;
+                    imp[mt][j] = 0.f;
+                }
+            }
         }
     }
 }
@@ -728,16 +733,20 @@ __global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_cons
             }
             n_loaded = first + n_tiles;
         }
+        if (ok && (p.per_head || g == p.Hkv - 1)) {
+            // the keys' scores are complete: of this KV group alone, or summed over all of them
+            float *out = p.scores + (p.per_head ? (int64_t)grp : (int64_t)lb) * p.Nv;
+#pragma unroll
+            for (int t = 0; t < KT; ++t) {
+                const int key = key0 + t * 128 + tid;
+                if (t < n_tiles && key < p.Nv) out[key] = imp[t];
+                imp[t] = 0.f;
+            }
+        }
     }
     ok = !s_abort;
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 128);
-    if (!ok) return;
-#pragma unroll
-    for (int t = 0; t < KT; ++t) {
-        const int key = key0 + t * 128 + tid;
-        if (t < n_tiles && key < p.Nv) p.scores[(int64_t)lb * p.Nv + key] = imp[t];
-    }
 }
 
 template <int D, int NT>
@@ -844,6 +853,7 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.group_ticket = ws_ptr<uint32_t>(ws, w.group_ticket);
     p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
     p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
+    p.per_head = s->per_kv_head;
     p.lb0 = layer_begin * s->batch;
     p.n_lb = layer_count * s->batch;
     p.cap = score_row_cap(s);

@@ -16,18 +16,21 @@ class Session:
         self.sh, self.ratio, self.alpha = sh, ratio, alpha
         self.dev = torch.device(device)
         L, B, Hq, Hkv, d, Nv = sh.n_layers, sh.batch, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.n_visual
-        LB = L * B
+        cells = Hkv if sh.per_kv_head else 1      # units with a budget of their own per (layer, sequence)
+        row_heads = 1 if sh.per_kv_head else Hkv  # KV heads stored in one row of the compressed cache
+        LB = L * B * cells
+        per = (cells,) if sh.per_kv_head else ()
         with torch.cuda.device(self.dev):
             self.ws = torch.empty(aircache_workspace_bytes(sh), dtype=torch.uint8, device=self.dev)
             aircache_reset_status(self.ws)
-        self.scores = torch.empty((L, B, Nv), dtype=torch.float32, device=self.dev)
+        self.scores = torch.empty((L, B) + per + (Nv,), dtype=torch.float32, device=self.dev)
         self.mask = torch.zeros((L, B, Hq), dtype=torch.int64, device=self.dev)
-        self.budgets = torch.empty((L, B), dtype=torch.int32, device=self.dev)
-        self.strength = torch.empty((L, B), dtype=torch.float64, device=self.dev)
-        self.skew = torch.empty((L, B), dtype=torch.float64, device=self.dev)
+        self.budgets = torch.empty((L, B) + per, dtype=torch.int32, device=self.dev)
+        self.strength = torch.empty((L, B) + per, dtype=torch.float64, device=self.dev)
+        self.skew = torch.empty((L, B) + per, dtype=torch.float64, device=self.dev)
         self.rows = aircache_total_rows(sh, ratio)
         self.kept_n = B * aircache_kept_per_sequence(sh, ratio)
-        self.k_c = torch.empty((self.rows, Hkv, d), dtype=torch.bfloat16, device=self.dev)
+        self.k_c = torch.empty((self.rows, row_heads, d), dtype=torch.bfloat16, device=self.dev)
         self.v_c = torch.empty_like(self.k_c)
         self.offsets = torch.zeros(LB + 1, dtype=torch.int64, device=self.dev)
         self.lens = torch.zeros(LB, dtype=torch.int32, device=self.dev)

@@ -44,10 +44,11 @@ def u16(t: torch.Tensor) -> np.ndarray:
 class GpuPath(Session):
     """Device buffers of one workload and the four stages as methods (thin calls into the C ABI)."""
 
-    def __init__(self, wl, ratio=None, device="cuda:0", slack=None):
+    def __init__(self, wl, ratio=None, device="cuda:0", slack=None, per_kv_head=0):
         self.wl = wl
         self.slack = wl.slack if slack is None else slack
-        super().__init__(shape_of(wl, slack=self.slack), wl.ratio if ratio is None else ratio, wl.alpha, device)
+        super().__init__(shape_of(wl, slack=self.slack, per_kv_head=per_kv_head), wl.ratio if ratio is None else ratio,
+                         wl.alpha, device)
 
 
 def gen_inputs(wl, device):

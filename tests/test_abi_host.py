@@ -4,6 +4,7 @@ import ctypes as C
 import os
 import re
 
+import numpy as np
 import pytest
 
 import paper_2503_23956_b200 as ac
@@ -25,7 +26,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(handle, n), f"{n} declared in aircache.h but not exported"
     assert sorted(ac.exported_symbols()) == names, "binding and header disagree"
-    assert ac.aircache_version() == 100
+    assert ac.aircache_version() == 101
 
 
 def test_strerror_covers_all_codes():
@@ -61,6 +62,14 @@ def test_shape_validation():
         sh = ac.shape(**{**good, **change})
         assert ac.aircache_workspace_bytes(sh) == code, change
         assert ac.aircache_total_rows(sh, 0.5) == code, change
+    # per-KV-head mode: every (layer, sequence, KV head) cell is a region of its own
+    per = ac.shape(**{**good, "per_kv_head": 1, "slack": 3})
+    Hkv, L, B = good["n_kv_heads"], good["n_layers"], good["batch"]
+    T = ac.aircache_kept_per_sequence(per, 0.3)
+    assert T == int(np.floor(0.3 * good["n_visual"] * L * Hkv + 0.5))
+    assert ac.aircache_total_rows(per, 0.3) == B * (T + L * Hkv * (good["n_text"] + 3))
+    assert ac.aircache_workspace_bytes(ac.shape(**{**good, "per_kv_head": 2})) == ac.ERR_INVALID_ARG
+    assert ac.aircache_workspace_bytes(ac.shape(**{**good, "per_kv_head": 1, "n_layers": 1792 // (B * Hkv) + 1})) == ac.ERR_UNSUPPORTED
     assert ac.aircache_total_rows(ac.shape(**good), 1.5) == ac.ERR_INVALID_ARG
     assert ac.aircache_total_rows(ac.shape(**good), float("nan")) == ac.ERR_INVALID_ARG
 

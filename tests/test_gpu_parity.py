@@ -419,6 +419,91 @@ def test_system_prompt_prefix_as_leading_text_rows(oracle):
     assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
 
 
+@pytest.mark.parametrize("case,alpha", [("s7b", 0.9), ("s72b", 0.9), ("c1", 0.9), ("kv2", 0.0), ("mha64", 0.9), ("g16", 0.9)])
+def test_per_kv_head_budgets_whole_chain(oracle, case, alpha):
+    """Per-KV-head mode: Eq. 8 averaged over a KV group's heads, Eq. 9-11 over the (layer, KV head) cells of a
+    sequence, every cell's own top-k and stretch of the ragged cache, decode and the fused append - against the
+    per-KV-group oracle.  Integer results equal, scores and outputs within 2e-3."""
+    import paper_2503_23956_b200 as ac
+    wl = CASES[case]
+    slack = 2
+    k, v, qw = cpu_inputs(wl)
+    dm = oracle_dims(oracle, wl)
+    kl, vl = u16(logical(k)), u16(logical(v))
+    sc = oracle.score_groups(dm, kl, u16(qw), wl.scale, alpha)
+    st, sk = oracle.moments(sc["scores"])
+    bud = oracle.allocate_groups(st, sk, wl.n_visual, wl.ratio)
+    cp = oracle.compact_groups(dm, slack, kl, vl, sc["scores"], bud)
+    assert (bud.sum(axis=(0, 2)) == oracle.total_kept(wl.n_visual, wl.n_layers * wl.n_kv_heads, wl.ratio)).all()
+
+    gp = GpuPath(wl, device=DEV, slack=slack, per_kv_head=1)
+    gp.set_full(logical(k.to(DEV)), logical(v.to(DEV)))
+    gp.score(qw.to(DEV), alpha=alpha)
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), sc["elite_mask"])
+    assert rel_elem_err(gp.scores.cpu().numpy(), sc["scores"]) <= TOL
+    # integer stages on the oracle's score bits, then the chained CUDA path
+    sc_d = torch.from_numpy(sc["scores"]).to(DEV)
+    gp.budget(scores=sc_d)
+    assert np.array_equal(gp.budgets.cpu().numpy(), bud)
+    assert np.allclose(gp.strength.cpu().numpy(), st, rtol=1e-12, atol=0)
+    assert np.allclose(gp.skew.cpu().numpy(), sk, rtol=1e-9, atol=1e-12)
+    gp.compact(scores=sc_d)
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+    gp.k_c.fill_(float("nan")); gp.v_c.fill_(float("nan"))
+    gp.budget()
+    gp.compact()
+    assert gp.status() == 0
+    assert np.array_equal(gp.budgets.cpu().numpy(), bud)
+    assert np.array_equal(gp.kept.cpu().numpy()[:len(cp["kept_idx"])], cp["kept_idx"])
+    compare_cache(gp, cp)
+    # decode: every query head attends to the cell of its KV head
+    gdm = oracle.group_decode_dims(dm)
+    cells, G = wl.n_layers * wl.batch * wl.n_kv_heads, wl.group
+    q = decode_queries(wl, 0, "cpu")
+    want = oracle.decode(gdm, cp["k"], cp["v"], cp["offsets"], cp["lens"], u16(q).reshape(cells, 1, G, wl.head_dim),
+                         wl.scale).reshape(q.shape)
+    gp.out.fill_(float("nan"))
+    gp.decode(q.to(DEV))
+    assert gp.status() == 0
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+    # Eq. 2 fused: one new row per cell
+    rng = np.random.default_rng(3)
+    kn = torch.from_numpy(rng.standard_normal((cells, 1, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+    vn = torch.from_numpy(rng.standard_normal((cells, 1, wl.head_dim)).astype(np.float32)).to(torch.bfloat16)
+    k_o, v_o, lens = cp["k"].copy(), cp["v"].copy(), cp["lens"].copy()
+    for c in range(cells):
+        k_o[cp["offsets"][c] + lens[c]] = u16(kn)[c]
+        v_o[cp["offsets"][c] + lens[c]] = u16(vn)[c]
+    lens += 1
+    q1 = decode_queries(wl, 1, "cpu")
+    want = oracle.decode(gdm, k_o, v_o, cp["offsets"], lens, u16(q1).reshape(cells, 1, G, wl.head_dim),
+                         wl.scale).reshape(q1.shape)
+    ac.aircache_decode_step(gp.sh, gp.cache, q1.to(DEV), kn.to(DEV), vn.to(DEV), 0, gp.out, gp.ws)
+    assert gp.status() == 0
+    assert np.array_equal(gp.lens.cpu().numpy(), lens)
+    assert rel_row_err(gp.out.cpu().numpy(), want) <= TOL
+    ac.aircache_append(gp.sh, gp.cache, kn.to(DEV), vn.to(DEV), 1)
+    assert np.array_equal(gp.lens.cpu().numpy(), lens + 1)
+
+
+def test_per_kv_head_with_one_kv_head_is_the_per_layer_method(oracle):
+    """With a single KV head the cells are the regions: the flag changes nothing, bit for bit."""
+    wl = CASES["kv1"]
+    ref = oracle_path(oracle, wl)
+    outs = []
+    for flag in (0, 1):
+        gp = GpuPath(wl, device=DEV, per_kv_head=flag)
+        gp.set_full(logical(ref["k"].to(DEV)), logical(ref["v"].to(DEV)))
+        run_chain(gp, ref)
+        gp.decode(decode_queries(wl, 0, DEV))
+        outs.append([t.cpu().numpy().reshape(-1).copy()
+                     for t in (gp.scores, gp.budgets, gp.kept, gp.k_c.view(torch.int16), gp.out)])
+    for a, b in zip(*outs):
+        assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
+    assert np.array_equal(outs[0][1].reshape(ref["budgets"].shape), ref["budgets"])
+
+
 def test_results_are_bit_reproducible(oracle):
     wl = CASES["s7b"]
     ref = oracle_path(oracle, wl)
