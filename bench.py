@@ -94,9 +94,9 @@ def pick_workload(spec: str, ratio, alpha=None):
     return wl
 
 
-def shape_of(ac, wl):
+def shape_of(ac, wl, per_kv_head=0):
     return ac.shape(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.n_visual, wl.n_text,
-                    wl.window, wl.slack, wl.scale)
+                    wl.window, wl.slack, wl.scale, per_kv_head)
 
 
 def logical(t):
@@ -184,7 +184,7 @@ def decode_cu_sha1():
     return hashlib.sha1(open(p, "rb").read()).hexdigest()[:12]
 
 
-def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, append=False):
+def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, append=False, per_kv_head=0):
     """Times `steps` steps of the whole path on `rotate` resident request batches of workload `wl`.
     Returns (local numbers, the sessions) -- the caller reduces over ranks."""
     from paper_2503_23956_b200.session import Session
@@ -192,7 +192,7 @@ def measure(ac, wl, n_dec, rotate, steps, warmup, use_graph, dev, rank, dist, ap
 
     if append:
         wl = wl.with_(slack=n_dec)   # room for one appended token per decode round (Eq. 2)
-    sh = shape_of(ac, wl)
+    sh = shape_of(ac, wl, per_kv_head)
     reqs = []
     for i in range(rotate):
         w = wl.with_(seed=wl.seed + 1000 * rank + i)
@@ -393,6 +393,92 @@ def workload_report(ac, spec, dev, rank, use_graph):
     return rep
 
 
+def per_kv_head_report(ac, spec, dev, rank, use_graph):
+    """The same workload with a budget and a kept set per (layer, sequence, KV head) (aircache_shape_t.per_kv_head):
+    stage times, decode time per call, and how far the KV heads' budget vectors over the layers lie from the
+    shared one (Jensen-Shannon divergence, bits)."""
+    wl = pick_workload(spec, None)
+    rot, _ = default_rotate(ac, wl)
+    d = min(wl.steps, 64)
+    m, q = measure(ac, wl, d, rot, 3, 3, use_graph, dev, rank, None, per_kv_head=1)
+    s = q[0]
+    bud = s.budgets[:, 0].cpu().numpy().astype(np.float64)          # [L, Hkv], sequence 0
+    shared = bud.sum(axis=1)
+
+    def js(a, b):
+        pa, pb = a / max(a.sum(), 1.0), b / max(b.sum(), 1.0)
+        mid = 0.5 * (pa + pb)
+        kl = lambda x, y: float(np.sum(x[x > 0] * np.log2(x[x > 0] / y[x > 0])))
+        return 0.5 * kl(pa, mid) + 0.5 * kl(pb, mid)
+
+    rep = {"workload": describe(wl) + " per_kv_head=1", "decode_steps": d, "resident_requests": rot,
+           "stage_us_per_request": {k: v * 1e3 / rot for k, v in m["stage_ms"].items()},
+           "decode_us_per_call": m["stage_ms"]["decode"] * 1e3 / (rot * d),
+           "budgets_sequence0_layer_by_kv_head": bud.astype(int).tolist(),
+           "js_divergence_bits_of_each_kv_head_vs_their_sum": [js(bud[:, g], shared) for g in range(bud.shape[1])]}
+    del q
+    return rep
+
+
+def per_layer_scoring(ac, spec, dev):
+    """Algorithm 1's first loop the way an engine runs it: after each layer's keys have been written (here: copied
+    into place, which leaves them in L2 as a prefill kernel would) aircache_score_layers scores that layer -
+    against one aircache_score call over the finished cache.  Same scores up to rounding."""
+    from paper_2503_23956_b200.session import Session
+    from workloads import full_cache, window_queries
+    wl = pick_workload(spec, None)
+    sh = shape_of(ac, wl)
+    s = Session(sh, wl.ratio, wl.alpha, dev)
+    k = full_cache(wl, "k", dev)
+    staging = k.clone()
+    s.set_full(logical(k), logical(k))
+    qw = window_queries(wl, dev)
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def timed(fn, reps=5):
+        """Average time (us) of fn's work, replayed as a CUDA graph of its C-ABI calls and copies."""
+        with torch.cuda.stream(stream):
+            fn()
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    def one_call():
+        s.score(qw, stream=stream)
+
+    def layer_by_layer(with_copy=True):
+        for l in range(wl.n_layers):
+            if with_copy:
+                k[l].copy_(staging[l])
+            ac.aircache_score_layers(sh, s.full, qw, wl.alpha, l, 1, s.scores, s.mask, s.ws, stream)
+
+    def copies_only():
+        for l in range(wl.n_layers):
+            k[l].copy_(staging[l])
+
+    with torch.cuda.stream(stream):
+        one_call()
+        want = s.scores.clone()
+        layer_by_layer()
+        stream.synchronize()
+    same = float(((want - s.scores).abs() / want.abs().clamp_min(1e-30)).max().item())
+    t_one, t_copy, t_both = timed(one_call), timed(copies_only), timed(layer_by_layer)
+    return {"workload": describe(wl), "one_call_us": t_one, "layer_by_layer_after_the_layers_write_us": t_both - t_copy,
+            "layer_writes_alone_us": t_copy, "max_rel_difference": same,
+            "key_mb_per_layer": wl.batch * wl.n_visual * wl.n_kv_heads * wl.head_dim * 2 / 1e6,
+            "note": "CUDA graph replay in all cases; a layer's keys fit in L2"}
+
+
 def run_cuda(args):
     import paper_2503_23956_b200 as ac
 
@@ -469,6 +555,10 @@ def run_cuda(args):
             "note": "aircache_decode_step (Eq. 2 append fused into the attention launch) per round and request"}
         result["score_dense_window"] = dense_window_score(w2, q3[0])
         del q3
+        torch.cuda.empty_cache()
+        result["per_kv_head"] = per_kv_head_report(ac, "c2", dev, rank, not args.no_graph)
+        torch.cuda.empty_cache()
+        result["score_layer_by_layer"] = per_layer_scoring(ac, "c4", dev)
         torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, n_dec)

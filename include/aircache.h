@@ -185,9 +185,11 @@ int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, c
  * aircache_budget once after the last layer.  All arrays are the ones
  * aircache_score takes (indexed by absolute layer); only the given layers' keys
  * and window queries are read and only their rows of scores / elite_mask are
- * written.  The result for a layer is bit-identical to what aircache_score
- * gives for it, whatever the split into ranges.  Calls that share a workspace
- * must be ordered on one stream.  layer_count = 0 is a no-op.
+ * written.  A layer's scores equal those of aircache_score up to rounding
+ * (into how many chunks a call cuts the keys, hence the order in which their
+ * softmax statistics merge, depends on how many layers it covers); equal calls
+ * give equal bits.  Calls that share a workspace must be ordered on one
+ * stream.  layer_count = 0 is a no-op.
  */
 int aircache_score_layers(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window,
                           float alpha, int32_t layer_begin, int32_t layer_count, float *scores,

@@ -54,7 +54,6 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     const int64_t LB = (int64_t)s->n_layers * s->batch;
     const int64_t groups = LB * s->n_kv_heads;
     const int64_t cap = score_row_cap(s);
-    const int64_t chunks = score_chunks(s);
     int64_t off = 0;
     auto take = [&](int64_t bytes) {
         int64_t at = off;
@@ -68,7 +67,7 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.row_info = take(groups * cap * 4);
     w.row_coef = take(groups * cap * 4);
     w.row_text = take(groups * cap * 8);
-    w.chunk_stats = take(groups * chunks * cap * 8);
+    w.chunk_stats = take(score_chunk_cells(s) * cap * 8);
     w.row_final = take(groups * cap * 8);
     w.group_ticket = take(groups * 4);
     w.mom_strength = take(n_cells(s) * 8);

@@ -75,23 +75,34 @@ inline int score_row_cap(const aircache_shape_t *s) {
     return (int)align_up((int64_t)g * s->window, 16);
 }
 
-// Visual-key chunks of the statistics pass.  592 CTAs run at a time on a B200 (four CTAs of 128 threads per
-// SM); a CTA costs about as much fixed time (row table, query staging, reduction, ticket) as streaming 600
-// keys.  The chunk count minimises waves * (fixed + keys per chunk) under at least 256 keys per chunk.  A
-// function of the shape only, so results are reproducible.
-inline int score_chunks(const aircache_shape_t *s) {
-    const int64_t groups = (int64_t)s->n_layers * s->batch * s->n_kv_heads;
-    int64_t most = s->n_visual / 256;
+// Visual-key chunks of the statistics pass for a call that covers `groups` KV groups (a range of layers).  592
+// CTAs run at a time on a B200 (four CTAs of 128 threads per SM); a CTA costs about as much fixed time (row
+// table, query staging, reduction, ticket) as streaming 600 keys.  The chunk count minimises
+// waves * (fixed + keys per chunk) under at least 256 keys per chunk.  A function of the shape and of the number
+// of layers the call covers only, so results are reproducible.
+inline int score_chunks(int n_visual, int64_t groups) {
+    int64_t most = n_visual / 256;
     if (most > 64) most = 64;
     if (most < 1) most = 1;
     int best = 1;
     int64_t best_cost = -1;
     for (int c = 1; c <= most; ++c) {
         const int64_t waves = (groups * c + 591) / 592;
-        const int64_t cost = waves * (600 + (s->n_visual + c - 1) / c);
+        const int64_t cost = waves * (600 + (n_visual + c - 1) / c);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = c; }
     }
     return best;
+}
+
+// The most (group, chunk) cells of statistics any call on this shape can have (it sizes the workspace).
+inline int64_t score_chunk_cells(const aircache_shape_t *s) {
+    int64_t most = 0;
+    for (int layers = 1; layers <= s->n_layers; ++layers) {
+        const int64_t groups = (int64_t)layers * s->batch * s->n_kv_heads;
+        const int64_t cells = groups * score_chunks(s->n_visual, groups);
+        if (cells > most) most = cells;
+    }
+    return most;
 }
 
 struct WsLayout {
@@ -102,7 +113,7 @@ struct WsLayout {
     int64_t row_info;     // i32  [L*B*Hkv][cap]       (head within group << 8) | window slot
     int64_t row_coef;     // f32  [L*B*Hkv][cap]       1 / (|E_h| * Hq)
     int64_t row_text;     // f32x2[L*B*Hkv][cap]       (max, sum) of the visible elite text logits, log2 domain
-    int64_t chunk_stats;  // f32x2[L*B*Hkv][chunks][cap]  (max, sum) over one chunk of visual keys
+    int64_t chunk_stats;  // f32x2[groups of the call][chunks][cap]  (max, sum) over one chunk of visual keys
     int64_t row_final;    // f32x2[L*B*Hkv][cap]       (max, weight / normaliser) after all chunks
     int64_t group_ticket; // u32  [L*B*Hkv]            chunks of the group done so far
     int64_t mom_strength; // f64  [cells]

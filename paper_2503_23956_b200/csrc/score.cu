@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
     const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
     const int n_rows = p.row_count[grp];
     if (n_rows <= p.rows_lo || n_rows > p.rows_hi) return;
-    float2 *out = p.chunk_stats + ((int64_t)grp * p.chunks + chunk) * p.cap;
+    float2 *out = p.chunk_stats + ((int64_t)(grp - p.lb0 * p.Hkv) * p.chunks + chunk) * p.cap;
 
     for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
         const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(128) stats_kernel(ScoreParams p) {
             mm = tx.x; zz = tx.y;
         }
         for (int c = lane; c < p.chunks; c += 32) {
-            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)grp * p.chunks + c) * p.cap + r);
+            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)(grp - p.lb0 * p.Hkv) * p.chunks + c) * p.cap + r);
             merge_stats(mm, zz, cs.x, cs.y);
         }
 #pragma unroll
@@ -535,7 +535,7 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
     const int key0 = chunk * p.chunk_keys, key1 = min(p.Nv, key0 + p.chunk_keys);
     const int n_tiles = key1 > key0 ? (key1 - key0 + 127) / 128 : 0;
     const int n_rows = p.row_count[grp];
-    float2 *out = p.chunk_stats + ((int64_t)grp * p.chunks + chunk) * p.cap;
+    float2 *out = p.chunk_stats + ((int64_t)(grp - p.lb0 * p.Hkv) * p.chunks + chunk) * p.cap;
 
     if (tid == 0) {
         for (int i = 0; i <= C::NST; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
@@ -627,7 +627,7 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
             mm = tx.x; zz = tx.y;
         }
         for (int c = lane; c < p.chunks; c += 32) {
-            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)grp * p.chunks + c) * p.cap + r);
+            const float2 cs = __ldcg(p.chunk_stats + ((int64_t)(grp - p.lb0 * p.Hkv) * p.chunks + c) * p.cap + r);
             merge_stats(mm, zz, cs.x, cs.y);
         }
 #pragma unroll
@@ -857,7 +857,7 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.lb0 = layer_begin * s->batch;
     p.n_lb = layer_count * s->batch;
     p.cap = score_row_cap(s);
-    p.chunks = score_chunks(s);
+    p.chunks = score_chunks(s->n_visual, (int64_t)layer_count * s->batch * s->n_kv_heads);
     p.chunk_keys = (int)align_up((s->n_visual + p.chunks - 1) / p.chunks, 16);
     p.scale = s->scale;
     p.sl2 = s->scale * kLog2e;

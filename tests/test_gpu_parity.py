@@ -356,7 +356,8 @@ def test_full_retention_equals_full_cache_decode(oracle):
 @pytest.mark.parametrize("case,alpha", [("s7b", 0.9), ("s7b", 0.0), ("c1", 0.9), ("many", 0.9)])
 def test_scoring_layer_by_layer_equals_one_call(oracle, case, alpha):
     """Algorithm 1's first loop taken a layer (or a few layers) at a time: aircache_score_layers over any split of
-    the layers writes the same bits as one aircache_score call, and those match the oracle."""
+    the layers gives the same elite sets and, up to the rounding of a different chunking of the keys, the same
+    scores as one aircache_score call; both match the oracle; equal calls give equal bits."""
     import paper_2503_23956_b200 as ac
     wl = CASES[case]
     ref = oracle_path(oracle, wl, alpha=alpha)
@@ -370,11 +371,17 @@ def test_scoring_layer_by_layer_equals_one_call(oracle, case, alpha):
         for begin, count in ranges:
             ac.aircache_score_layers(gp.sh, gp.full, qw, alpha, begin, count, gp.scores, gp.mask, gp.ws)
         assert gp.status() == 0
-        assert torch.equal(gp.scores, whole) and torch.equal(gp.mask, whole_mask)
-    # a single layer leaves the other layers' rows alone
+        assert torch.equal(gp.mask, whole_mask)
+        assert rel_elem_err(gp.scores.cpu().numpy(), whole.cpu().numpy()) <= 1e-5
+        assert rel_elem_err(gp.scores.cpu().numpy(), ref["scores"]) <= TOL
+    # a single layer leaves the other layers' rows alone, and the same call twice gives the same bits
     gp.scores.fill_(float("nan"))
     ac.aircache_score_layers(gp.sh, gp.full, qw, alpha, L - 1, 1, gp.scores, gp.mask, gp.ws)
-    assert torch.isnan(gp.scores[:L - 1]).all() and torch.equal(gp.scores[L - 1], whole[L - 1])
+    assert torch.isnan(gp.scores[:L - 1]).all()
+    last = gp.scores[L - 1].clone()
+    assert rel_elem_err(last.cpu().numpy(), whole[L - 1].cpu().numpy()) <= 1e-5
+    ac.aircache_score_layers(gp.sh, gp.full, qw, alpha, L - 1, 1, gp.scores, gp.mask, gp.ws)
+    assert torch.equal(gp.scores[L - 1], last)
     assert np.array_equal(whole_mask.cpu().numpy().view(np.uint64), ref["mask"])
     assert rel_elem_err(whole.cpu().numpy(), ref["scores"]) <= TOL
 
