@@ -479,6 +479,41 @@ def per_layer_scoring(ac, spec, dev):
             "note": "CUDA graph replay in all cases; a layer's keys fit in L2"}
 
 
+def window_sweep(ac, spec, dev, windows=(16, 64, 128)):
+    """aircache_score with the candidate window W = the last 16 / 64 / all 128 text tokens of the workload (the
+    paper's own window is all of them), at the paper's threshold and with every candidate kept (alpha = 0: the
+    continuous-window variants of its ablation, computed by the tcgen05 kernels)."""
+    from paper_2503_23956_b200.session import Session
+    from workloads import full_cache, window_queries
+    wl0 = pick_workload(spec, None)
+    k = full_cache(wl0, "k", dev)
+    out = {}
+    for W in windows:
+        if W > wl0.n_text:
+            continue
+        wl = wl0.with_(window=W)
+        s = Session(shape_of(ac, wl), wl.ratio, wl.alpha, dev)
+        s.set_full(logical(k), logical(k))
+        qw = window_queries(wl, dev)
+        row = {}
+        for alpha in (wl.alpha, 0.0):
+            for _ in range(3):
+                s.score(qw, alpha=alpha)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                s.score(qw, alpha=alpha)
+            e1.record()
+            torch.cuda.synchronize()
+            bits = s.mask.cpu().numpy().view(np.uint8)
+            rows = float(np.unpackbits(bits).sum()) / (wl.n_layers * wl.batch * wl.n_kv_heads)
+            row[f"alpha_{alpha:g}"] = {"score_us": e0.elapsed_time(e1) * 1e2, "elite_rows_per_kv_group": rows}
+        out[f"W{W}"] = row
+        del s
+    return {"workload": describe(wl0), "windows": out, "note": "direct C-ABI calls, one resident request"}
+
+
 def run_cuda(args):
     import paper_2503_23956_b200 as ac
 
@@ -555,6 +590,8 @@ def run_cuda(args):
             "note": "aircache_decode_step (Eq. 2 append fused into the attention launch) per round and request"}
         result["score_dense_window"] = dense_window_score(w2, q3[0])
         del q3
+        torch.cuda.empty_cache()
+        result["window_sweep"] = window_sweep(ac, "c2", dev)
         torch.cuda.empty_cache()
         result["per_kv_head"] = per_kv_head_report(ac, "c2", dev, rank, not args.no_graph)
         torch.cuda.empty_cache()

@@ -73,7 +73,8 @@ typedef struct {
     int32_t head_dim;    /* d in {64, 128}                                                           */
     int32_t n_visual;    /* Nv >= 3 visual tokens per sequence (Eq. 10 needs three)                  */
     int32_t n_text;      /* Nt >= 1 text tokens per sequence                                         */
-    int32_t window;      /* W: the last W text tokens are the candidates of Eq. 5; 1 <= W <= min(64, Nt) */
+    int32_t window;      /* W: the last W text tokens are the candidates of Eq. 5; 1 <= W <= min(128, Nt);
+                            W = Nt is the paper's window (every text token a candidate)                */
     int32_t slack;       /* rows left free after each region for tokens appended while decoding, >= 0 */
     float scale;         /* softmax scale of Eq. 4 and Eq. 7, normally 1 / sqrt(head_dim)            */
     int32_t per_kv_head; /* 0: one budget and one kept set per (layer, sequence), shared by all KV heads
@@ -170,7 +171,8 @@ int64_t aircache_workspace_bytes(const aircache_shape_t *shape);
  *                                      text token Nt-W+w; the last one is the reference of Eq. 4)
  *   alpha       relevance threshold in [0, 1]
  *   scores      fp32 [L, B, Nv]        output I_v
- *   elite_mask  u64  [L, B, Hq]        output, bit w set <=> candidate w is elite; may be NULL
+ *   elite_mask  u64  [L, B, Hq, ceil(W/64)]  output, candidate w is elite <=> bit w % 64 of word w / 64 is
+ *                                      set (one word per head up to W = 64, two beyond); may be NULL
  */
 int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window,
                    float alpha, float *scores, uint64_t *elite_mask, void *workspace, int64_t workspace_bytes,

@@ -85,6 +85,12 @@ def full_cache_strides(k: np.ndarray) -> tuple[int, int, int, int]:
     return s[0], s[1], s[2], s[3]
 
 
+def _mask_shape(dims: Dims):
+    """Elite masks: one 64-bit word per query head, two when the window has more than 64 candidates."""
+    words = (dims.window + 63) // 64
+    return (dims.n_layers, dims.batch, dims.n_q_heads) + ((words,) if words > 1 else ())
+
+
 def score(dims: Dims, k: np.ndarray, q_window: np.ndarray, scale: float, alpha: float,
           want_logits: bool = False):
     """Eq. 4-8.  k: uint16 logical [L,B,Hkv,N,d] (any strides, d contiguous); q_window: uint16 [L,B,W,Hq,d].
@@ -97,7 +103,7 @@ def score(dims: Dims, k: np.ndarray, q_window: np.ndarray, scale: float, alpha: 
     assert q_window.shape == (L, B, W, Hq, dims.head_dim), q_window.shape
     sl, sb, sh, st = full_cache_strides(k)
     scores = np.empty((L, B, dims.n_visual), np.float32)
-    mask = np.empty((L, B, Hq), np.uint64)
+    mask = np.empty(_mask_shape(dims), np.uint64)
     tmass = np.empty((L, B, Hq), np.float64)
     logits = np.empty((L, B, Hq, W), np.float32) if want_logits else None
     d = dims.c()
@@ -121,7 +127,7 @@ def score_groups(dims: Dims, k: np.ndarray, q_window: np.ndarray, scale: float, 
     assert q_window.shape == (L, B, W, Hq, dims.head_dim), q_window.shape
     sl, sb, sh, st = full_cache_strides(k)
     scores = np.empty((L, B, dims.n_kv_heads, dims.n_visual), np.float32)
-    mask = np.empty((L, B, Hq), np.uint64)
+    mask = np.empty(_mask_shape(dims), np.uint64)
     d = dims.c()
     rc = lib().oracle_score_groups(C.byref(d), _p(k), C.c_int64(sl), C.c_int64(sb), C.c_int64(sh), C.c_int64(st),
                                    _p(q_window), C.c_float(scale), C.c_float(alpha), _p(scores), _p(mask))

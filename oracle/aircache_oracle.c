@@ -62,12 +62,14 @@ static double dot_bf16(const uint16_t *a, const uint16_t *b, int d) {
  * CUDA path states for it: the fp64 dot product is rounded to fp32, scaled in
  * fp32, and the difference to the maximum is compared in fp32 with
  * (float)log((double)alpha).  alpha = 0 keeps every candidate.
- * Returns a W-bit mask (bit w set <=> candidate w is elite); logits_out (may be
- * NULL) receives the W fp32 logits.
+ * Returns a W-bit mask (bit w set <=> candidate w is elite; W <= 128); logits_out
+ * (may be NULL) receives the W fp32 logits.
  */
-static uint64_t elite_of_head(const uint16_t *q_last, const uint16_t *k_cand0, int64_t k_stride_token,
-                              int W, int d, float scale, float alpha, float *logits_out) {
-    float t[64];
+typedef unsigned __int128 mask128_t;   /* one bit per candidate, W <= 128 */
+
+static mask128_t elite_of_head(const uint16_t *q_last, const uint16_t *k_cand0, int64_t k_stride_token,
+                               int W, int d, float scale, float alpha, float *logits_out) {
+    float t[128];
     float tmax = -INFINITY;
     for (int w = 0; w < W; ++w) {
         float dotf = (float)dot_bf16(q_last, k_cand0 + (int64_t)w * k_stride_token, d);
@@ -75,15 +77,15 @@ static uint64_t elite_of_head(const uint16_t *q_last, const uint16_t *k_cand0, i
         if (t[w] > tmax) tmax = t[w];
         if (logits_out) logits_out[w] = t[w];
     }
-    uint64_t mask = 0;
+    mask128_t mask = 0;
     if (alpha <= 0.0f) {
-        for (int w = 0; w < W; ++w) mask |= (uint64_t)1 << w;
+        for (int w = 0; w < W; ++w) mask |= (mask128_t)1 << w;
         return mask;
     }
     float ln_alpha = (float)log((double)alpha);
     for (int w = 0; w < W; ++w) {
         float diff = t[w] - tmax;
-        if (diff >= ln_alpha) mask |= (uint64_t)1 << w;
+        if (diff >= ln_alpha) mask |= (mask128_t)1 << w;
     }
     return mask;
 }
@@ -93,7 +95,7 @@ static uint64_t elite_of_head(const uint16_t *q_last, const uint16_t *k_cand0, i
  *   k            bf16 full key cache, strides in elements
  *   q_window     bf16 [L, B, W, Hq, d] contiguous: queries of the W candidate text tokens
  *   scores       fp32 [L, B, Nv]      (output)  I_v, rounded to fp32 once at the end
- *   elite_mask   u64  [L, B, Hq]      (output, may be NULL)
+ *   elite_mask   u64  [L, B, Hq, ceil(W/64)]  (output, may be NULL) candidate w is bit w % 64 of word w / 64
  *   text_mass    f64  [L, B, Hq]      (output, may be NULL) mean over elite rows of the
  *                                     softmax mass that fell on text keys (for the sum-to-one pin)
  *   elite_logits fp32 [L, B, Hq, W]   (output, may be NULL) the Eq. 4 logits the decision used
@@ -134,7 +136,8 @@ static int score_worker(const oracle_dims_t *dm, const uint16_t *k, int64_t s_la
                         float *group_scores) {
     const int L = dm->n_layers, B = dm->batch, Hq = dm->n_q_heads, Hkv = dm->n_kv_heads;
     const int d = dm->head_dim, Nv = dm->n_visual, Nt = dm->n_text, W = dm->window;
-    if (W < 1 || W > 64 || W > Nt || Hq % Hkv != 0 || Nv < 1) return -1;
+    if (W < 1 || W > 128 || W > Nt || Hq % Hkv != 0 || Nv < 1) return -1;
+    const int words = (W + 63) / 64;
     const int G = Hq / Hkv;
     const int N = Nv + Nt;
     int status = 0;
@@ -155,9 +158,11 @@ static int score_worker(const oracle_dims_t *dm, const uint16_t *k, int64_t s_la
                 const uint16_t *k_g = k_lb + (int64_t)g * s_head;
                 const uint16_t *q_last = q_lb + ((int64_t)(W - 1) * Hq + h) * d;
                 float *lg = elite_logits ? elite_logits + (((int64_t)l * B + b) * Hq + h) * W : NULL;
-                uint64_t E = elite_of_head(q_last, k_g + (int64_t)(N - W) * s_token, s_token, W, d, scale,
-                                           alpha, lg);
-                if (elite_mask) elite_mask[((int64_t)l * B + b) * Hq + h] = E;
+                mask128_t E = elite_of_head(q_last, k_g + (int64_t)(N - W) * s_token, s_token, W, d, scale,
+                                            alpha, lg);
+                if (elite_mask)
+                    for (int j = 0; j < words; ++j)
+                        elite_mask[(((int64_t)l * B + b) * Hq + h) * words + j] = (uint64_t)(E >> (64 * j));
                 int n_elite = 0;
                 for (int w = 0; w < W; ++w) n_elite += (int)((E >> w) & 1);
                 for (int i = 0; i < Nv; ++i) per_head[i] = 0.0;
@@ -171,7 +176,7 @@ static int score_worker(const oracle_dims_t *dm, const uint16_t *k, int64_t s_la
                         logit[i] = (double)scale * dot_bf16(q_w, k_g + (int64_t)i * s_token, d);
                         if (logit[i] > m) m = logit[i];
                     }
-                    double tl[64];
+                    double tl[128];
                     for (int w2 = 0; w2 <= w; ++w2) {
                         if (!((E >> w2) & 1)) continue;
                         tl[w2] = (double)scale * dot_bf16(q_w, k_g + (int64_t)(N - W + w2) * s_token, d);

@@ -9,7 +9,7 @@
 
 namespace aircache {
 
-constexpr int kMaxWindow = 64;
+constexpr int kMaxWindow = 128;
 constexpr int kMaxGroup = 16;         // query heads per KV head
 constexpr int kMaxRegions = 1792;     // L * B (the decode kernel keeps the unit prefix of all regions in shared memory)
 constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)

@@ -65,8 +65,9 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     uint16_t *s_k = s_dyn;                 // [W][KS]   candidate keys
     uint16_t *s_ql = s_dyn + p.W * KS;     // [G][KS]   queries of the last text token
     __shared__ float s_logit[kMaxGroup * kMaxWindow];
-    __shared__ uint64_t s_mask[kMaxGroup];
+    __shared__ uint64_t s_mask[kMaxGroup][2];   // candidate w is bit w % 64 of word w / 64
     __shared__ int s_first_row[kMaxGroup + 1];
+    const int words = (p.W + 63) >> 6;
 
     const int grp = p.lb0 * p.Hkv + blockIdx.x;  // (l*B + b)*Hkv + g
     const int g = grp % p.Hkv;
@@ -112,20 +113,22 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         const float *t = s_logit + hl * p.W;
         float tmax = -INFINITY;
         for (int w = 0; w < p.W; ++w) tmax = fmaxf(tmax, t[w]);
-        uint64_t mask = 0;
+        uint64_t mask[2] = {0, 0};
         for (int w = 0; w < p.W; ++w) {
             const float diff = __fsub_rn(t[w], tmax);
-            if (p.keep_all || diff >= p.ln_alpha) mask |= (uint64_t)1 << w;
+            if (p.keep_all || diff >= p.ln_alpha) mask[w >> 6] |= (uint64_t)1 << (w & 63);
         }
-        s_mask[hl] = mask;
-        if (p.elite_mask) p.elite_mask[(int64_t)lb * p.Hq + g * p.G + hl] = mask;
+        s_mask[hl][0] = mask[0];
+        s_mask[hl][1] = mask[1];
+        if (p.elite_mask)
+            for (int j = 0; j < words; ++j) p.elite_mask[((int64_t)lb * p.Hq + g * p.G + hl) * words + j] = mask[j];
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         int r = 0;
         for (int hl = 0; hl < p.G; ++hl) {
             s_first_row[hl] = r;
-            r += __popcll(s_mask[hl]);
+            r += __popcll(s_mask[hl][0]) + __popcll(s_mask[hl][1]);
         }
         s_first_row[p.G] = r;
         p.row_count[grp] = r;
@@ -138,11 +141,15 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     float2 *text = p.row_text + (int64_t)grp * p.cap;
     for (int idx = threadIdx.x; idx < p.G * p.W; idx += blockDim.x) {
         const int hl = idx / p.W, w = idx % p.W;
-        const uint64_t mask = s_mask[hl];
-        if (!((mask >> w) & 1)) continue;
-        const int r = s_first_row[hl] + __popcll(mask & (((uint64_t)1 << w) - 1));
+        const uint64_t m_lo = s_mask[hl][0], m_hi = s_mask[hl][1];
+        auto elite = [&](int j) { return (((j < 64 ? m_lo : m_hi) >> (j & 63)) & 1) != 0; };
+        if (!elite(w)) continue;
+        // elite candidates in front of w
+        const int before = w < 64 ? __popcll(m_lo & (((uint64_t)1 << w) - 1))
+                                  : __popcll(m_lo) + __popcll(m_hi & (((uint64_t)1 << (w - 64)) - 1));
+        const int r = s_first_row[hl] + before;
         info[r] = (hl << 8) | w;
-        coef[r] = 1.0f / ((float)__popcll(mask) * (float)(p.per_head ? p.G : p.Hq));
+        coef[r] = 1.0f / ((float)(__popcll(m_lo) + __popcll(m_hi)) * (float)(p.per_head ? p.G : p.Hq));
         // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.  The query row goes to registers
         // once, the keys come from shared memory.
         uint4 qr[D / 8];
@@ -151,7 +158,7 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
-            if (!((mask >> w2) & 1)) continue;
+            if (!elite(w2)) continue;
             const uint4 *kk = reinterpret_cast<const uint4 *>(s_k + w2 * KS);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll

@@ -24,7 +24,8 @@ class Session:
             self.ws = torch.empty(aircache_workspace_bytes(sh), dtype=torch.uint8, device=self.dev)
             aircache_reset_status(self.ws)
         self.scores = torch.empty((L, B) + per + (Nv,), dtype=torch.float32, device=self.dev)
-        self.mask = torch.zeros((L, B, Hq), dtype=torch.int64, device=self.dev)
+        words = (sh.window + 63) // 64
+        self.mask = torch.zeros((L, B, Hq) + ((words,) if words > 1 else ()), dtype=torch.int64, device=self.dev)
         self.budgets = torch.empty((L, B) + per, dtype=torch.int32, device=self.dev)
         self.strength = torch.empty((L, B) + per, dtype=torch.float64, device=self.dev)
         self.skew = torch.empty((L, B) + per, dtype=torch.float64, device=self.dev)

@@ -56,7 +56,7 @@ def test_shape_validation():
         (dict(scale=0.0), ac.ERR_INVALID_ARG), (dict(scale=float("nan")), ac.ERR_INVALID_ARG),
         (dict(head_dim=96), ac.ERR_UNSUPPORTED), (dict(n_kv_heads=3, n_q_heads=6), ac.ERR_UNSUPPORTED),
         (dict(n_q_heads=64, n_kv_heads=2), ac.ERR_UNSUPPORTED), (dict(n_visual=2), ac.ERR_UNSUPPORTED),
-        (dict(n_text=80, window=65), ac.ERR_UNSUPPORTED), (dict(n_layers=64, batch=64), ac.ERR_UNSUPPORTED),
+        (dict(n_text=200, window=129), ac.ERR_UNSUPPORTED), (dict(n_layers=64, batch=64), ac.ERR_UNSUPPORTED),
     ]
     for change, code in bad:
         sh = ac.shape(**{**good, **change})

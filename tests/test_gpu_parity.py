@@ -29,6 +29,9 @@ CASES = {
     "g16": small("g16", L=2, Hq=16, Hkv=1, d=64, B=2, Nv=257, Nt=17, W=5),   # 16 query heads per KV head
     "kv2": small("kv2", L=2, Hq=12, Hkv=2, d=128, B=2, Nv=515, Nt=64, W=64),  # widest window
     "kv1": small("kv1", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=130, Nt=9, W=9),
+    # the paper's own window: every text token a candidate (W = N_t = 128: two mask words per head)
+    "w128": small("w128", L=2, Hq=28, Hkv=4, d=128, B=1, Nv=700, Nt=128, W=128),
+    "w100": small("w100", L=1, Hq=8, Hkv=2, d=64, B=2, Nv=300, Nt=100, W=100),
     # long regions cut across many CTAs with an odd head count (padded partial slots, multi-round merge)
     "kv1long": small("kv1long", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=9000, Nt=9, W=4, ratio=0.9),
     # more (region, KV head) pairs than SMs: the by-region decode schedule with several regions per CTA
@@ -104,7 +107,7 @@ def test_score_parity(oracle, case, alpha):
     assert err <= TOL, err
 
 
-@pytest.mark.parametrize("case", ["kv2", "s7b", "g16"])
+@pytest.mark.parametrize("case", ["kv2", "s7b", "g16", "w128"])
 def test_score_parity_many_elite_rows_below_the_dense_threshold(oracle, case):
     """A small but non-zero threshold makes almost every candidate elite (hundreds of rows per KV group on the
     widest window) while the launch stays on the sparse-window kernels: their loops over slabs of rows run more
@@ -308,7 +311,7 @@ def run_chain(gp, ref):
     gp.compact()
 
 
-@pytest.mark.parametrize("case", ["c1", "s7b", "s72b", "kv2", "maxreg"])
+@pytest.mark.parametrize("case", ["c1", "s7b", "s72b", "kv2", "maxreg", "w128"])
 def test_end_to_end_chain(oracle, case):
     wl = CASES[case]
     ref = oracle_path(oracle, wl)

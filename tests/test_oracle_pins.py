@@ -92,6 +92,36 @@ def test_elite_matches_literal_softmax_threshold(oracle_mod):
         assert checked > 20
 
 
+def test_window_of_all_text_tokens_beyond_64(oracle_mod):
+    """The paper's own window: every text token is a candidate (W = N_t, here 100 > 64, so the elite set takes two
+    mask words).  Eq. 5 literally on the library softmax row, and Eq. 6-8 in matrix form on that set."""
+    rng = np.random.default_rng(5)
+    L, B, Hq, Hkv, d, Nv, Nt = 1, 2, 4, 2, 32, 19, 100
+    W = Nt
+    k, _, qw = rand_case(rng, L, B, Hq, Hkv, d, Nv, Nt, W)
+    dm = oracle_mod.Dims(L, B, Hq, Hkv, d, Nv, Nt, W)
+    scale = 1 / math.sqrt(d)
+    kf, qf = bf16_val(k), bf16_val(qw)
+    for alpha in (0.0, 0.5, 0.9):
+        out = oracle_mod.score(dm, k, qw, scale, alpha)
+        assert out["elite_mask"].shape == (L, B, Hq, 2)
+        for l, b in itertools.product(range(L), range(B)):
+            acc = np.zeros(Nv)
+            for h in range(Hq):
+                g = h // (Hq // Hkv)
+                E = int(out["elite_mask"][l, b, h, 0]) | int(out["elite_mask"][l, b, h, 1]) << 64
+                a = torch.softmax(torch.from_numpy(kf[l, b, g, Nv:, :] @ qf[l, b, W - 1, h, :] * scale), 0).numpy()
+                rel = a / a.max()
+                if np.abs(rel - alpha).min() > 1e-4:
+                    assert E == sum(1 << j for j in range(W) if rel[j] >= alpha)
+                assert E >> W == 0 and E >> int(np.argmax(a)) & 1
+                iv, _ = literal_importance(kf[l, b, g], qf[l, b, :, h, :], E, Nv, Nt, W, scale)
+                acc += iv
+            assert np.allclose(out["scores"][l, b], acc / Hq, rtol=2e-7, atol=0)
+        if alpha == 0.0:
+            assert (out["elite_mask"][..., 0] == 2 ** 64 - 1).all() and (out["elite_mask"][..., 1] == 2 ** 36 - 1).all()
+
+
 # ----------------------------------------------------------------------------------------------
 # Eq. 6-8: inter-modal attention and importance
 # ----------------------------------------------------------------------------------------------
