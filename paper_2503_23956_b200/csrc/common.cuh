@@ -94,9 +94,16 @@ inline int score_chunks(int n_visual, int64_t groups) {
     return best;
 }
 
+// One-pass scoring (both passes of Eq. 7 in one block, logits kept on chip between them): a block covers
+// 64 * tiles keys of one KV group, tiles = 16 / (row tiles of the group) in {4, 8, 16}; the grid is laid out for
+// the smallest block, 256 keys; the largest is 1024.
+constexpr int kOnePassMinKeys = 256;
+constexpr int kOnePassMaxKeys = 1024;
+inline int onepass_chunks(int n_visual) { return (n_visual + kOnePassMinKeys - 1) / kOnePassMinKeys; }
+
 // The most (group, chunk) cells of statistics any call on this shape can have (it sizes the workspace).
 inline int64_t score_chunk_cells(const aircache_shape_t *s) {
-    int64_t most = 0;
+    int64_t most = (int64_t)s->n_layers * s->batch * s->n_kv_heads * onepass_chunks(s->n_visual);
     for (int layers = 1; layers <= s->n_layers; ++layers) {
         const int64_t groups = (int64_t)layers * s->batch * s->n_kv_heads;
         const int64_t cells = groups * score_chunks(s->n_visual, groups);
@@ -116,6 +123,9 @@ struct WsLayout {
     int64_t chunk_stats;  // f32x2[groups of the call][chunks][cap]  (max, sum) over one chunk of visual keys
     int64_t row_final;    // f32x2[L*B*Hkv][cap]       (max, weight / normaliser) after all chunks
     int64_t group_ticket; // u32  [L*B*Hkv]            chunks of the group done so far
+    int64_t dispatch;     // u32                       blocks of the one-pass scoring kernel started so far
+    int64_t imp_part;     // f32  [L*B*Hkv][Nv]        importance of one KV group before the sum over groups
+    int64_t q_block;      // bf16 [L*B*Hkv][32][d]     the first 32 elite query rows of a group, gathered
     int64_t mom_strength; // f64  [cells]
     int64_t mom_skew;     // f64  [cells]
     int64_t kept;         // i32  [cells*Nv]           kept-token lists when the caller passes none

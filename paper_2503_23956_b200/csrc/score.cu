@@ -19,6 +19,7 @@
 // Both passes read the keys straight from global memory into MMA fragments: every key byte is used once
 // per CTA, so staging it in shared memory would only add a round trip.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -40,6 +41,10 @@ struct ScoreParams {
     float2 *chunk_stats;
     float2 *row_final;   // (max, weight / normaliser) per elite row, written by the last stats CTA of a group
     uint32_t *group_ticket;
+    uint32_t *dispatch;     // one-pass scoring: blocks started so far
+    float *imp_part;        // one-pass scoring: [L*B*Hkv][Nv] importance of one KV group
+    uint16_t *q_block;      // one-pass scoring: [L*B*Hkv][32][d] the first 32 elite query rows, gathered
+    int op_chunks;
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
     int lb0, n_lb;   // the launch covers regions lb0 .. lb0 + n_lb - 1 (a range of layers)
     int per_head;    // scores are kept apart per KV group: [L,B,Hkv,Nv], Eq. 8 averaged over the group's heads only
@@ -78,7 +83,10 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
     const uint16_t *k_cand = k_g + (int64_t)(N - p.W) * p.s_token;
     const uint16_t *q_lb = p.qw + (int64_t)lb * p.W * p.Hq * D;
 
-    if (threadIdx.x == 0) p.group_ticket[grp] = 0;   // the statistics pass counts its chunks here
+    if (threadIdx.x == 0) {
+        p.group_ticket[grp] = 0;   // the statistics pass counts its chunks here
+        if (blockIdx.x == 0) *p.dispatch = 0;
+    }
     for (int idx = threadIdx.x; idx < (p.W + p.G) * (D / 8); idx += blockDim.x) {
         const int row = idx / (D / 8), c = idx % (D / 8);
         const uint16_t *src = row < p.W ? k_cand + (int64_t)row * p.s_token
@@ -156,6 +164,11 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         const uint4 *qq = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D);
 #pragma unroll
         for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
+        if (r < 32) {   // the one-pass kernel stages the first 32 rows from this gathered copy
+            uint4 *qb = reinterpret_cast<uint4 *>(p.q_block + ((int64_t)grp * 32 + r) * D);
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) qb[c] = qr[c];
+        }
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
             if (!elite(w2)) continue;
@@ -212,6 +225,25 @@ __device__ __forceinline__ void tile_mma(float (&acc)[4], const KeyFrag<D> &f, c
         mma_bf16_16816(acc, f.lo[kb].x, f.hi[kb].x, f.lo[kb].y, f.hi[kb].y, bq.x, bq.y);
         mma_bf16_16816(acc, f.lo[kb].z, f.hi[kb].z, f.lo[kb].w, f.hi[kb].w, bq.z, bq.w);
     }
+}
+
+// The same tile with the contraction split over two accumulators (channels 0..d/2-1 and d/2..d-1) that are
+// added at the end: half the dependent-MMA chain, for callers with few row tiles to interleave.
+template <int D>
+__device__ __forceinline__ void tile_mma_split(float (&acc)[4], const KeyFrag<D> &f, const uint16_t *q_row, int t) {
+    constexpr int H = D / 64;
+    float lo[4] = {0.f, 0.f, 0.f, 0.f}, hi[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int kb = 0; kb < H; ++kb) {
+        const uint4 bq = *reinterpret_cast<const uint4 *>(q_row + kb * 32 + 8 * t);
+        const uint4 bq2 = *reinterpret_cast<const uint4 *>(q_row + (kb + H) * 32 + 8 * t);
+        mma_bf16_16816(lo, f.lo[kb].x, f.hi[kb].x, f.lo[kb].y, f.hi[kb].y, bq.x, bq.y);
+        mma_bf16_16816(hi, f.lo[kb + H].x, f.hi[kb + H].x, f.lo[kb + H].y, f.hi[kb + H].y, bq2.x, bq2.y);
+        mma_bf16_16816(lo, f.lo[kb].z, f.hi[kb].z, f.lo[kb].w, f.hi[kb].w, bq.z, bq.w);
+        mma_bf16_16816(hi, f.lo[kb + H].z, f.hi[kb + H].z, f.lo[kb + H].w, f.hi[kb + H].w, bq2.z, bq2.w);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = lo[i] + hi[i];
 }
 
 // Copies up to 8*NT elite query rows (starting at row0) of one KV group into shared memory, zero padded.
@@ -437,6 +469,289 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
             }
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 7 and Eq. 8 in ONE pass over the keys.
+//
+// The two kernels above read the keys from HBM twice when the cache is larger than L2.  Here a block owns a
+// chunk of one KV group's keys and keeps the chunk's logits (fp32 MMA accumulators, up to 32 rows) in shared
+// memory: pass one gives the chunk's (max, sum) per row; when all chunks of the group have published theirs,
+// every block of the group merges them (same fixed order in every block: equal bits), turns its stored logits
+// into probabilities and sums them per key - no second read of the keys, no second contraction.  A chunk is
+// 64 * tiles keys with tiles = 16 / (row tiles of the group), so the stored logits always fill the same 32 KB;
+// rows beyond 32 (wide windows, small alpha) are recomputed from the keys, which are still in L1/L2.
+//
+// Waiting inside a grid is safe here because a block draws its number from a counter when it STARTS: all
+// lower numbers belong to blocks that are running or done.  Numbers are group-major, a group spans
+// op_chunks numbers, and the host only takes this path when op_chunks is at most half of the blocks the GPU
+// holds at once - so the blocks a waiting block depends on are always resident or next in line, and blocks
+// of lower groups, which wait for nothing that has not started, always finish.  The wait is bounded all the same.
+//
+// The sum over the KV groups of a (layer, sequence) is a second, small kernel (fixed order g = 0, 1, ...).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *ptr) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ int onepass_tiles(int n_rows) {   // 16-key tiles per warp
+    const int nt0 = (n_rows + 7) >> 3;
+    return nt0 <= 1 ? 16 : (nt0 == 2 ? 8 : 4);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
+    constexpr int NT = 4, QS = D + 32;
+    extern __shared__ __align__(16) uint16_t s_dyn[];
+    float4 *s_S = reinterpret_cast<float4 *>(s_dyn);        // [tile of the warp][row tile][thread]: 2048 x 16 B
+    __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
+    __shared__ float2 s_red[4][NT * 8];
+    __shared__ float2 s_stat[NT * 8];
+    __shared__ float s_imp[kOnePassMaxKeys];
+    __shared__ int s_flag;
+
+    if (threadIdx.x == 0) s_flag = (int)atomicAdd(p.dispatch, 1u);
+    __syncthreads();
+    const int vid = s_flag;
+    __syncthreads();
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gid = lane >> 2, t = lane & 3;
+    const int gi = vid / p.op_chunks, c = vid % p.op_chunks;
+    if (gi >= p.n_lb * p.Hkv) return;
+    const int grp = p.lb0 * p.Hkv + gi;
+    const int g = grp % p.Hkv, lb = grp / p.Hkv, l = lb / p.B, b = lb % p.B;
+    const int n_rows = p.row_count[grp];
+    const int tpw = onepass_tiles(n_rows);
+    const int KB = 64 * tpw;
+    const int chunks_g = (p.Nv + KB - 1) / KB;
+    if (c >= chunks_g) return;
+    const int nt0 = min(NT, (n_rows + 7) >> 3);
+    const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
+    const int key0 = c * KB, key1 = min(p.Nv, key0 + KB);
+    const int wk0 = key0 + warp * tpw * 16, wk1 = min(key1, wk0 + tpw * 16);
+    // the warp's whole key range is asked into L2 first: HBM latency runs beside the query staging
+    for (int i = lane; i < (wk1 - wk0) * (D * 2 / 128); i += 32)
+        prefetch_l2(k_g + (int64_t)(wk0 + i / (D * 2 / 128)) * p.s_token + (i % (D * 2 / 128)) * 64);
+
+    auto fetch = [&](KeyFrag<D> &dst, int kt) {
+        const int ka = kt + gid, kb = kt + gid + 8;
+        load_keys<D>(dst, k_g + (int64_t)(ka < wk1 ? ka : wk1 - 1) * p.s_token,
+                     k_g + (int64_t)(kb < wk1 ? kb : wk1 - 1) * p.s_token, t);
+    };
+    // (max, weight / normaliser) of rows row0 .. row0 + n - 1 into s_stat: one thread per row merges the text
+    // statistics and then the chunks' statistics in chunk order (all loads of a row are independent, one round
+    // trip), the same order in every block
+    auto merge_rows = [&](int row0, int n) {
+        if (tid < n) {
+            const int row = row0 + tid;
+            float2 fin = make_float2(0.f, 0.f);
+            if (row < n_rows) {
+                const float2 *cs = p.chunk_stats + (int64_t)gi * p.op_chunks * p.cap + row;
+                const float2 tx = p.row_text[(int64_t)grp * p.cap + row];
+                const float coef = p.row_coef[(int64_t)grp * p.cap + row];
+                float mm = tx.x, zz = tx.y;
+                int cc = 0;
+                for (; cc + 4 <= chunks_g; cc += 4) {
+                    const float2 c0 = __ldcg(cs + (int64_t)cc * p.cap), c1 = __ldcg(cs + (int64_t)(cc + 1) * p.cap);
+                    const float2 c2 = __ldcg(cs + (int64_t)(cc + 2) * p.cap), c3 = __ldcg(cs + (int64_t)(cc + 3) * p.cap);
+                    merge_stats(mm, zz, c0.x, c0.y); merge_stats(mm, zz, c1.x, c1.y);
+                    merge_stats(mm, zz, c2.x, c2.y); merge_stats(mm, zz, c3.x, c3.y);
+                }
+                for (; cc < chunks_g; ++cc) {
+                    const float2 c0 = __ldcg(cs + (int64_t)cc * p.cap);
+                    merge_stats(mm, zz, c0.x, c0.y);
+                }
+                fin = make_float2(mm, coef / zz);
+            }
+            s_stat[tid] = fin;
+        }
+    };
+
+    // ---- pass one: statistics of the chunk, logits of the first 32 rows kept ----
+    float2 *out = p.chunk_stats + ((int64_t)gi * p.op_chunks + c) * p.cap;
+    for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
+        const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
+        KeyFrag<D> f, f_next;
+        if (wk0 < wk1) fetch(f, wk0);
+        __syncthreads();
+        if (row0 == 0) {
+            const uint4 *qb = reinterpret_cast<const uint4 *>(p.q_block + (int64_t)grp * 32 * D);
+            for (int idx = tid; idx < nt_used * 8 * (D / 8); idx += blockDim.x) {
+                const int r = idx / (D / 8), cc = idx % (D / 8);
+                *reinterpret_cast<uint4 *>(s_q + r * QS + cc * 8) = r < n_rows ? __ldg(qb + idx) : make_uint4(0, 0, 0, 0);
+            }
+        } else {
+            stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
+        }
+        __syncthreads();
+        float m[NT][2], z[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { m[nt][0] = m[nt][1] = kNegBig; z[nt][0] = z[nt][1] = 0.f; }
+        int slot = tid;   // (tile * nt_used + nt) * 128 + tid
+        for (int kt = wk0; kt < wk1; kt += 16) {
+            const int ka = kt + gid, kb = kt + gid + 8;
+            const bool va = ka < wk1, vb = kb < wk1;
+            if (kt + 16 < wk1) fetch(f_next, kt + 16);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (nt < nt_used) {
+                    float acc[4];
+                    tile_mma_split<D>(acc, f, s_q + (nt * 8 + gid) * QS, t);
+                    if (row0 == 0) { s_S[slot] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot += 128; }
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const float xa = va ? acc[j] * p.sl2 : kNegBig;
+                        const float xb = vb ? acc[j + 2] * p.sl2 : kNegBig;
+                        const float mn = fmaxf(m[nt][j], fmaxf(xa, xb));
+                        const float ea = va ? fast_exp2(xa - mn) : 0.f;
+                        const float eb = vb ? fast_exp2(xb - mn) : 0.f;
+                        z[nt][j] = z[nt][j] * fast_exp2(m[nt][j] - mn) + (ea + eb);
+                        m[nt][j] = mn;
+                    }
+                }
+            }
+            if (kt + 16 < wk1) f = f_next;
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            if (nt < nt_used) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    float mm = m[nt][j], zz = z[nt][j];
+#pragma unroll
+                    for (int sh = 4; sh < 32; sh <<= 1) {
+                        const float m2 = __shfl_xor_sync(0xffffffffu, mm, sh);
+                        const float z2 = __shfl_xor_sync(0xffffffffu, zz, sh);
+                        merge_stats(mm, zz, m2, z2);
+                    }
+                    if (gid == 0) s_red[warp][nt * 8 + 2 * t + j] = make_float2(mm, zz);
+                }
+            }
+        }
+        __syncthreads();
+        for (int r = tid; r < nt_used * 8; r += blockDim.x) {
+            float2 a = s_red[0][r];
+#pragma unroll
+            for (int w2 = 1; w2 < 4; ++w2) merge_stats(a.x, a.y, s_red[w2][r].x, s_red[w2][r].y);
+            if (row0 + r < n_rows) __stcg(out + row0 + r, a);
+        }
+    }
+
+    // ---- publish the chunk, wait until every chunk of the group is published ----
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();   // the block's statistics (ordered before this by the barrier) before the ticket
+        int ok = atomicAdd(p.group_ticket + grp, 1u) + 1u >= (unsigned)chunks_g;
+        for (uint32_t i = 0; !ok && i < kSpinLimit; ++i) {
+            __nanosleep(i < 64 ? 32 : 1000);
+            ok = ld_acquire_u32(p.group_ticket + grp) >= (unsigned)chunks_g;
+        }
+        if (!ok) atomicExch(p.status, 8u);
+        __threadfence();
+        s_flag = ok;
+    }
+    __syncthreads();
+    if (!s_flag) return;
+
+    // ---- pass two: probabilities from the kept logits, summed over the rows of the group ----
+    merge_rows(0, nt0 * 8);
+    __syncthreads();
+    {
+        int slot = tid, at = warp * tpw * 16;
+#pragma unroll 4
+        for (int kt = wk0; kt < wk1; kt += 16, at += 16) {
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (nt < nt0) {
+                    const float4 v = s_S[slot]; slot += 128;
+                    const float2 s0 = s_stat[nt * 8 + 2 * t], s1 = s_stat[nt * 8 + 2 * t + 1];
+                    a0 += fast_exp2(v.x * p.sl2 - s0.x) * s0.y + fast_exp2(v.y * p.sl2 - s1.x) * s1.y;
+                    a1 += fast_exp2(v.z * p.sl2 - s0.x) * s0.y + fast_exp2(v.w * p.sl2 - s1.x) * s1.y;
+                }
+            }
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+            if (t == 0) { s_imp[at + gid] = a0; s_imp[at + gid + 8] = a1; }
+        }
+    }
+    // rows beyond 32: logits recomputed from the keys
+    for (int row0 = NT * 8; row0 < n_rows; row0 += NT * 8) {
+        const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
+        __syncthreads();
+        stage_queries<D>(s_q, p, grp, lb, g, row0, n_rows, nt_used * 8);
+        merge_rows(row0, nt_used * 8);
+        __syncthreads();
+        KeyFrag<D> f;
+        int at = warp * tpw * 16;
+        for (int kt = wk0; kt < wk1; kt += 16, at += 16) {
+            fetch(f, kt);
+            float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                if (nt < nt_used) {
+                    float acc[4];
+                    tile_mma_split<D>(acc, f, s_q + (nt * 8 + gid) * QS, t);
+                    const float2 s0 = s_stat[nt * 8 + 2 * t], s1 = s_stat[nt * 8 + 2 * t + 1];
+                    a0 += fast_exp2(acc[0] * p.sl2 - s0.x) * s0.y + fast_exp2(acc[1] * p.sl2 - s1.x) * s1.y;
+                    a1 += fast_exp2(acc[2] * p.sl2 - s0.x) * s0.y + fast_exp2(acc[3] * p.sl2 - s1.x) * s1.y;
+                }
+            }
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+            if (t == 0) { s_imp[at + gid] += a0; s_imp[at + gid + 8] += a1; }
+        }
+    }
+    __syncthreads();
+
+    // ---- Eq. 8: the group's own score, or its part of the sum over the KV groups ----
+    const int nkeys = key1 - key0;
+    float *dst = (p.per_head ? p.scores : p.imp_part) + (int64_t)grp * p.Nv + key0;
+    for (int i = tid; i < nkeys; i += blockDim.x) dst[i] = s_imp[i];
+}
+
+// Eq. 8, the mean over all query heads: the KV groups' parts added in the order g = 0, 1, ...
+__global__ void __launch_bounds__(256) group_sum_kernel(ScoreParams p) {
+    const int lb = p.lb0 + blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.Nv) return;
+    const float *src = p.imp_part + (int64_t)lb * p.Hkv * p.Nv + i;
+    float v = 0.f;
+    for (int g = 0; g < p.Hkv; ++g) v += __ldcg(src + (int64_t)g * p.Nv);
+    p.scores[(int64_t)lb * p.Nv + i] = v;
+}
+
+// Blocks of the one-pass kernel the device holds at once (0 if the kernel cannot run); asked once per device.
+template <int D>
+int onepass_resident_blocks() {
+    static int cached[64];
+    static bool have[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!have[dev]) {
+        int per_sm = 0, sms = 0;
+        if (cudaFuncSetAttribute(onepass_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, onepass_kernel<D>, 128, 32768) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return 0;
+        cached[dev] = per_sm * sms;
+        have[dev] = true;
+    }
+    return cached[dev];
+}
+
+template <int D>
+int launch_onepass(const ScoreParams &p, cudaStream_t st) {
+    const int64_t blocks = (int64_t)p.n_lb * p.Hkv * p.op_chunks;
+    onepass_kernel<D><<<(unsigned)blocks, 128, 32768, st>>>(p);
+    AIRCACHE_LAUNCH_CHECK();
+    if (!p.per_head) {
+        group_sum_kernel<<<dim3((p.Nv + 255) / 256, (unsigned)p.n_lb), 256, 0, st>>>(p);
+        AIRCACHE_LAUNCH_CHECK();
+    }
+    return AIRCACHE_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -858,6 +1173,10 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.chunk_stats = ws_ptr<float2>(ws, w.chunk_stats);
     p.row_final = ws_ptr<float2>(ws, w.row_final);
     p.group_ticket = ws_ptr<uint32_t>(ws, w.group_ticket);
+    p.dispatch = ws_ptr<uint32_t>(ws, w.dispatch);
+    p.imp_part = ws_ptr<float>(ws, w.imp_part);
+    p.q_block = ws_ptr<uint16_t>(ws, w.q_block);
+    p.op_chunks = onepass_chunks(s->n_visual);
     p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
     p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
     p.per_head = s->per_kv_head;
@@ -888,6 +1207,14 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
             return s->head_dim == 64 ? launch_dense<64>(p, tm, st) : launch_dense<128>(p, tm, st);
     }
 #endif
+    // one pass over the keys, if a group's blocks are sure to be resident together
+    bool one = true;
+#ifdef AIRCACHE_SCORE_KNOBS
+    if (const char *e = getenv("AIRCACHE_ONEPASS_OFF")) one = atoi(e) == 0;
+#endif
+    const int resident = s->head_dim == 64 ? onepass_resident_blocks<64>() : onepass_resident_blocks<128>();
+    if (one && (int64_t)p.op_chunks * 2 <= resident && (int64_t)p.n_lb * p.Hkv * p.op_chunks < ((int64_t)1 << 31))
+        return s->head_dim == 64 ? launch_onepass<64>(p, st) : launch_onepass<128>(p, st);
     return s->head_dim == 64 ? launch_passes_d<64>(p, st) : launch_passes_d<128>(p, st);
 }
 
