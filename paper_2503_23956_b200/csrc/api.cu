@@ -72,7 +72,7 @@ WsLayout ws_layout(const aircache_shape_t *s) {
     w.group_ticket = take(groups * 4);
     w.dispatch = take(256);
     w.imp_part = take(s->per_kv_head ? 256 : groups * (int64_t)s->n_visual * 4);
-    w.q_block = take(groups * 32 * (int64_t)s->head_dim * 2);
+    w.q_block = take(groups * 16 * (int64_t)s->head_dim * 2);
     w.mom_strength = take(n_cells(s) * 8);
     w.mom_skew = take(n_cells(s) * 8);
     w.kept = take(n_cells(s) * s->n_visual * 4);

@@ -94,10 +94,9 @@ inline int score_chunks(int n_visual, int64_t groups) {
     return best;
 }
 
-// One-pass scoring (both passes of Eq. 7 in one block, logits kept on chip between them): a block covers
-// 64 * tiles keys of one KV group, tiles = 16 / (row tiles of the group) in {4, 8, 16}; the grid is laid out for
-// the smallest block, 256 keys; the largest is 1024.
-constexpr int kOnePassMinKeys = 256;
+// One-pass scoring (both passes of Eq. 7 in one block, logits kept on chip between them): a block covers 1024
+// keys of a KV group with up to 8 elite rows, 512 keys otherwise; the grid is laid out for 512.
+constexpr int kOnePassMinKeys = 512;
 constexpr int kOnePassMaxKeys = 1024;
 inline int onepass_chunks(int n_visual) { return (n_visual + kOnePassMinKeys - 1) / kOnePassMinKeys; }
 
@@ -125,7 +124,7 @@ struct WsLayout {
     int64_t group_ticket; // u32  [L*B*Hkv]            chunks of the group done so far
     int64_t dispatch;     // u32                       blocks of the one-pass scoring kernel started so far
     int64_t imp_part;     // f32  [L*B*Hkv][Nv]        importance of one KV group before the sum over groups
-    int64_t q_block;      // bf16 [L*B*Hkv][32][d]     the first 32 elite query rows of a group, gathered
+    int64_t q_block;      // bf16 [L*B*Hkv][16][d]     the first 16 elite query rows of a group, gathered
     int64_t mom_strength; // f64  [cells]
     int64_t mom_skew;     // f64  [cells]
     int64_t kept;         // i32  [cells*Nv]           kept-token lists when the caller passes none

@@ -19,7 +19,6 @@
 // Both passes read the keys straight from global memory into MMA fragments: every key byte is used once
 // per CTA, so staging it in shared memory would only add a round trip.
 #include <math.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "ptx.cuh"
@@ -43,7 +42,7 @@ struct ScoreParams {
     uint32_t *group_ticket;
     uint32_t *dispatch;     // one-pass scoring: blocks started so far
     float *imp_part;        // one-pass scoring: [L*B*Hkv][Nv] importance of one KV group
-    uint16_t *q_block;      // one-pass scoring: [L*B*Hkv][32][d] the first 32 elite query rows, gathered
+    uint16_t *q_block;      // one-pass scoring: [L*B*Hkv][16][d] the first 16 elite query rows, gathered
     int op_chunks;
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
     int lb0, n_lb;   // the launch covers regions lb0 .. lb0 + n_lb - 1 (a range of layers)
@@ -164,8 +163,8 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         const uint4 *qq = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D);
 #pragma unroll
         for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
-        if (r < 32) {   // the one-pass kernel stages the first 32 rows from this gathered copy
-            uint4 *qb = reinterpret_cast<uint4 *>(p.q_block + ((int64_t)grp * 32 + r) * D);
+        if (r < 16) {   // the one-pass kernel stages the first 16 rows from this gathered copy
+            uint4 *qb = reinterpret_cast<uint4 *>(p.q_block + ((int64_t)grp * 16 + r) * D);
 #pragma unroll
             for (int c = 0; c < D / 8; ++c) qb[c] = qr[c];
         }
@@ -475,12 +474,13 @@ __global__ void __launch_bounds__(128) importance_kernel(ScoreParams p) {
 // Eq. 7 and Eq. 8 in ONE pass over the keys.
 //
 // The two kernels above read the keys from HBM twice when the cache is larger than L2.  Here a block owns a
-// chunk of one KV group's keys and keeps the chunk's logits (fp32 MMA accumulators, up to 32 rows) in shared
+// chunk of one KV group's keys and keeps the chunk's logits (fp32 MMA accumulators, up to 16 rows) in shared
 // memory: pass one gives the chunk's (max, sum) per row; when all chunks of the group have published theirs,
 // every block of the group merges them (same fixed order in every block: equal bits), turns its stored logits
 // into probabilities and sums them per key - no second read of the keys, no second contraction.  A chunk is
-// 64 * tiles keys with tiles = 16 / (row tiles of the group), so the stored logits always fill the same 32 KB;
-// rows beyond 32 (wide windows, small alpha) are recomputed from the keys, which are still in L1/L2.
+// 1024 keys for a group of up to 8 elite rows and 512 keys beyond, so the stored logits fill the same 32 KB
+// (five blocks per SM); the per-key sums of pass two go into slots of that buffer the warp has already read.
+// Rows beyond 16 (wide windows, small alpha) are recomputed from the keys, which are still in L1/L2.
 //
 // Waiting inside a grid is safe here because a block draws its number from a counter when it STARTS: all
 // lower numbers belong to blocks that are running or done.  Numbers are group-major, a group spans
@@ -497,19 +497,17 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *ptr) {
 }
 
 __device__ __forceinline__ int onepass_tiles(int n_rows) {   // 16-key tiles per warp
-    const int nt0 = (n_rows + 7) >> 3;
-    return nt0 <= 1 ? 16 : (nt0 == 2 ? 8 : 4);
+    return n_rows <= 8 ? 16 : 8;
 }
 
 template <int D>
-__global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
-    constexpr int NT = 4, QS = D + 32;
+__global__ void __launch_bounds__(128, 5) onepass_kernel(ScoreParams p) {
+    constexpr int NT = 2, QS = D + 32;
     extern __shared__ __align__(16) uint16_t s_dyn[];
     float4 *s_S = reinterpret_cast<float4 *>(s_dyn);        // [tile of the warp][row tile][thread]: 2048 x 16 B
     __shared__ __align__(16) uint16_t s_q[NT * 8 * QS];
     __shared__ float2 s_red[4][NT * 8];
     __shared__ float2 s_stat[NT * 8];
-    __shared__ float s_imp[kOnePassMaxKeys];
     __shared__ int s_flag;
 
     if (threadIdx.x == 0) s_flag = (int)atomicAdd(p.dispatch, 1u);
@@ -569,7 +567,7 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
         }
     };
 
-    // ---- pass one: statistics of the chunk, logits of the first 32 rows kept ----
+    // ---- pass one: statistics of the chunk, logits of the first 16 rows kept ----
     float2 *out = p.chunk_stats + ((int64_t)gi * p.op_chunks + c) * p.cap;
     for (int row0 = 0; row0 < n_rows; row0 += NT * 8) {
         const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
@@ -577,7 +575,7 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
         if (wk0 < wk1) fetch(f, wk0);
         __syncthreads();
         if (row0 == 0) {
-            const uint4 *qb = reinterpret_cast<const uint4 *>(p.q_block + (int64_t)grp * 32 * D);
+            const uint4 *qb = reinterpret_cast<const uint4 *>(p.q_block + (int64_t)grp * 16 * D);
             for (int idx = tid; idx < nt_used * 8 * (D / 8); idx += blockDim.x) {
                 const int r = idx / (D / 8), cc = idx % (D / 8);
                 *reinterpret_cast<uint4 *>(s_q + r * QS + cc * 8) = r < n_rows ? __ldg(qb + idx) : make_uint4(0, 0, 0, 0);
@@ -659,9 +657,10 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
     merge_rows(0, nt0 * 8);
     __syncthreads();
     {
-        int slot = tid, at = warp * tpw * 16;
+        int slot = tid;
+        float *imp_w = reinterpret_cast<float *>(s_S + warp * 32);   // + tile * nt0 * 512 floats: the warp's own slots of the tile
 #pragma unroll 4
-        for (int kt = wk0; kt < wk1; kt += 16, at += 16) {
+        for (int kt = wk0; kt < wk1; kt += 16, imp_w += nt0 * 512) {
             float a0 = 0.f, a1 = 0.f;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
@@ -674,10 +673,10 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
             }
             a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
-            if (t == 0) { s_imp[at + gid] = a0; s_imp[at + gid + 8] = a1; }
+            if (t == 0) { imp_w[gid] = a0; imp_w[gid + 8] = a1; }
         }
     }
-    // rows beyond 32: logits recomputed from the keys
+    // rows beyond 16: logits recomputed from the keys
     for (int row0 = NT * 8; row0 < n_rows; row0 += NT * 8) {
         const int nt_used = min(NT, (n_rows - row0 + 7) / 8);
         __syncthreads();
@@ -685,8 +684,8 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
         merge_rows(row0, nt_used * 8);
         __syncthreads();
         KeyFrag<D> f;
-        int at = warp * tpw * 16;
-        for (int kt = wk0; kt < wk1; kt += 16, at += 16) {
+        float *imp_w = reinterpret_cast<float *>(s_S + warp * 32);
+        for (int kt = wk0; kt < wk1; kt += 16, imp_w += nt0 * 512) {
             fetch(f, kt);
             float a0 = 0.f, a1 = 0.f;
 #pragma unroll
@@ -701,7 +700,7 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
             }
             a0 += __shfl_xor_sync(0xffffffffu, a0, 1); a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 1); a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
-            if (t == 0) { s_imp[at + gid] += a0; s_imp[at + gid + 8] += a1; }
+            if (t == 0) { imp_w[gid] += a0; imp_w[gid + 8] += a1; }
         }
     }
     __syncthreads();
@@ -709,7 +708,10 @@ __global__ void __launch_bounds__(128, 4) onepass_kernel(ScoreParams p) {
     // ---- Eq. 8: the group's own score, or its part of the sum over the KV groups ----
     const int nkeys = key1 - key0;
     float *dst = (p.per_head ? p.scores : p.imp_part) + (int64_t)grp * p.Nv + key0;
-    for (int i = tid; i < nkeys; i += blockDim.x) dst[i] = s_imp[i];
+    for (int i = tid; i < nkeys; i += blockDim.x) {
+        const int w = i / (tpw * 16), rem = i % (tpw * 16);
+        dst[i] = reinterpret_cast<const float *>(s_S + w * 32)[(rem >> 4) * nt0 * 512 + (rem & 15)];
+    }
 }
 
 // Eq. 8, the mean over all query heads: the KV groups' parts added in the order g = 0, 1, ...
@@ -1208,12 +1210,8 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     }
 #endif
     // one pass over the keys, if a group's blocks are sure to be resident together
-    bool one = true;
-#ifdef AIRCACHE_SCORE_KNOBS
-    if (const char *e = getenv("AIRCACHE_ONEPASS_OFF")) one = atoi(e) == 0;
-#endif
     const int resident = s->head_dim == 64 ? onepass_resident_blocks<64>() : onepass_resident_blocks<128>();
-    if (one && (int64_t)p.op_chunks * 2 <= resident && (int64_t)p.n_lb * p.Hkv * p.op_chunks < ((int64_t)1 << 31))
+    if ((int64_t)p.op_chunks * 2 <= resident && (int64_t)p.n_lb * p.Hkv * p.op_chunks < ((int64_t)1 << 31))
         return s->head_dim == 64 ? launch_onepass<64>(p, st) : launch_onepass<128>(p, st);
     return s->head_dim == 64 ? launch_passes_d<64>(p, st) : launch_passes_d<128>(p, st);
 }

@@ -107,6 +107,21 @@ def test_score_parity(oracle, case, alpha):
     assert err <= TOL, err
 
 
+def test_score_parity_sequence_longer_than_the_one_pass_kernel_takes(oracle):
+    """The one-pass scoring kernel lets the blocks of a KV group wait for one another, so the library only uses
+    it while a group's blocks (one per 512 visual keys) are at most half of the blocks the GPU holds at once;
+    200 000 visual tokens are beyond that on any GPU of today (391 blocks per group against at most 370), and
+    the call takes the two-kernel form (statistics pass, then importance pass) instead."""
+    wl = small("verylong", L=1, Hq=2, Hkv=1, d=64, B=1, Nv=200_000, Nt=16, W=8)
+    ref = oracle_path(oracle, wl, alpha=0.9)
+    gp = make_gpu(wl, ref)
+    gp.score(ref["qw"].to(DEV), alpha=0.9)
+    assert gp.status() == 0
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64), ref["mask"]), "elite sets differ"
+    err = rel_elem_err(gp.scores.cpu().numpy(), ref["scores"])
+    assert err <= TOL, err
+
+
 @pytest.mark.parametrize("case", ["kv2", "s7b", "g16", "w128"])
 def test_score_parity_many_elite_rows_below_the_dense_threshold(oracle, case):
     """A small but non-zero threshold makes almost every candidate elite (hundreds of rows per KV group on the
