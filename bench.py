@@ -308,7 +308,7 @@ def rooflines(ac, wl, m, rotate, n_dec, traffic=None):
     comp = roof("select_kernel + gather_kernel per aircache_compact call", compact_bytes,
                 m["stage_ms"]["compact"] * 1e3 / rotate)
     score_bytes = LB * wl.n_visual * (row_bytes + 4)
-    score = roof("elite_kernel + stats_kernel + importance_kernel per aircache_score call", score_bytes,
+    score = roof("elite_kernel + onepass_kernel + group_sum_kernel per aircache_score call", score_bytes,
                  m["stage_ms"]["score"] * 1e3 / rotate)
     return dec, comp, score
 
@@ -321,10 +321,10 @@ def default_rotate(ac, wl):
 
 
 def kernels_per_step(wl, rotate, n_dec):
-    """Launches of this library's kernels in one step: elite + statistics (one launch, two when a KV group may
-    have more than 32 elite rows) + importance; budget; select + gather; one decode kernel per call."""
-    nt_max = (wl.group * wl.window + 7) // 8
-    score = 1 + (1 if nt_max <= 4 else 2) + 1
+    """Launches of this library's kernels in one step: elite + one-pass scoring + sum over the KV groups; budget;
+    select + gather; one decode kernel per call.  (alpha = 0 and sequences too long for the one-pass kernel
+    launch differently; no bench workload is either.)"""
+    score = 3
     return rotate * (score + 1 + 2 + n_dec)
 
 

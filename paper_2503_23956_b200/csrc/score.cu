@@ -63,7 +63,7 @@ constexpr float kNegBig = -1.0e30f;
 // Eq. 4-5 and the elite-row table
 // ---------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
+__global__ void __launch_bounds__(128, 6) elite_kernel(ScoreParams p) {
     constexpr int KS = D + 8;   // padded row: 16-byte reads of consecutive rows fall into different banks
     extern __shared__ __align__(16) uint16_t s_dyn[];
     uint16_t *s_k = s_dyn;                 // [W][KS]   candidate keys
@@ -106,8 +106,10 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
             const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                acc = __dadd_rn(acc, __dmul_rn((double)bf16lo(av[e]), (double)bf16lo(bv[e])));
-                acc = __dadd_rn(acc, __dmul_rn((double)bf16hi(av[e]), (double)bf16hi(bv[e])));
+                // a product of two bf16 values is exact in fp64, so the fused form rounds exactly where the
+                // separate multiply and add do
+                acc = __fma_rn((double)bf16lo(av[e]), (double)bf16lo(bv[e]), acc);
+                acc = __fma_rn((double)bf16hi(av[e]), (double)bf16hi(bv[e]), acc);
             }
         }
         s_logit[idx] = __fmul_rn((float)acc, p.scale);
@@ -157,25 +159,22 @@ __global__ void __launch_bounds__(128) elite_kernel(ScoreParams p) {
         const int r = s_first_row[hl] + before;
         info[r] = (hl << 8) | w;
         coef[r] = 1.0f / ((float)(__popcll(m_lo) + __popcll(m_hi)) * (float)(p.per_head ? p.G : p.Hq));
-        // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.  The query row goes to registers
-        // once, the keys come from shared memory.
-        uint4 qr[D / 8];
+        // Eq. 6-7, text columns: row w sees the elite text keys w' <= w.  The keys come from shared memory, the
+        // query row is re-read for every key (256 bytes that stay in L1) rather than held in 64 registers.
         const uint4 *qq = reinterpret_cast<const uint4 *>(q_lb + ((int64_t)w * p.Hq + g * p.G + hl) * D);
-#pragma unroll
-        for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
         if (r < 16) {   // the one-pass kernel stages the first 16 rows from this gathered copy
             uint4 *qb = reinterpret_cast<uint4 *>(p.q_block + ((int64_t)grp * 16 + r) * D);
-#pragma unroll
-            for (int c = 0; c < D / 8; ++c) qb[c] = qr[c];
+#pragma unroll 4
+            for (int c = 0; c < D / 8; ++c) qb[c] = __ldg(qq + c);
         }
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
             if (!elite(w2)) continue;
             const uint4 *kk = reinterpret_cast<const uint4 *>(s_k + w2 * KS);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
+#pragma unroll 4
             for (int c = 0; c < D / 8; ++c) {
-                const uint4 a = qr[c], bb = kk[c];
+                const uint4 a = __ldg(qq + c), bb = kk[c];
                 a0 = fmaf(bf16lo(a.x), bf16lo(bb.x), a0); a1 = fmaf(bf16hi(a.x), bf16hi(bb.x), a1);
                 a2 = fmaf(bf16lo(a.y), bf16lo(bb.y), a2); a3 = fmaf(bf16hi(a.y), bf16hi(bb.y), a3);
                 a0 = fmaf(bf16lo(a.z), bf16lo(bb.z), a0); a1 = fmaf(bf16hi(a.z), bf16hi(bb.z), a1);
