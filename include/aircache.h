@@ -49,7 +49,7 @@
 extern "C" {
 #endif
 
-#define AIRCACHE_VERSION 101
+#define AIRCACHE_VERSION 102
 
 #define AIRCACHE_OK 0
 #define AIRCACHE_ERR_INVALID_ARG (-1)          /* NULL pointer, negative size, ratio outside [0,1], ...        */
@@ -60,6 +60,7 @@ extern "C" {
 #define AIRCACHE_ERR_CUDA (-6)                 /* a CUDA call failed; see aircache_last_cuda_error()            */
 #define AIRCACHE_ERR_TIMEOUT (-7)              /* a bounded device-side wait gave up (aircache_check_status)    */
 #define AIRCACHE_ERR_STATIC_SCRATCH (-8)       /* aircache_decode_attn_static: built-in scratch array too small */
+#define AIRCACHE_ERR_INCONSISTENT (-9)         /* aircache_compact found budgets / offsets that do not fit the buffers (aircache_check_status) */
 
 /* Size of the device array that aircache_decode_attn_static uses as scratch, per GPU. */
 #define AIRCACHE_STATIC_SCRATCH_BYTES (12 * 1024 * 1024)
@@ -222,6 +223,13 @@ int aircache_budget(const aircache_shape_t *shape, const float *scores, double r
  * wins), then K' = Concat(K_v[kept], K_t), V' = Concat(V_v[kept], V_t) are
  * gathered into the region's rows, kept tokens in ascending token order.
  * out->offsets and out->lens must hold what aircache_budget wrote for `budgets`.
+ * Both live in device memory, so the host cannot check them: the kernels do.  A
+ * budget outside [0, Nv], a kept list that would leave the list buffer, a row
+ * that would land outside [0, out->total_rows) or a listed token outside
+ * [0, Nv) is not followed - the entries and rows concerned stay unwritten - and
+ * aircache_check_status() then reports AIRCACHE_ERR_INCONSISTENT.  (Values that
+ * fit the buffers but do not belong together, such as regions that overlap,
+ * cannot be told from a layout the caller meant.)
  *   ratio      the same ratio aircache_budget was given (sizes the launch; capacity check)
  *   kept_idx   i32, region r's ascending token list at position offsets[r] - r*(Nt+slack);
  *              B * T entries in total; may be NULL
@@ -303,13 +311,15 @@ int aircache_append(const aircache_shape_t *shape, aircache_ragged_t *cache, con
  * tickets and the plans that decode launches keep from one call to the next
  * (about 150 KB in all).  Must be called once after allocating the workspace,
  * before its first use by aircache_budget or aircache_decode_attn, and again
- * after an AIRCACHE_ERR_TIMEOUT.
+ * after an AIRCACHE_ERR_TIMEOUT or AIRCACHE_ERR_INCONSISTENT.
  */
 int aircache_reset_status(void *workspace, int64_t workspace_bytes, void *cuda_stream);
 
 /*
- * Synchronises the stream, reads the workspace's status word and returns 0 or
- * AIRCACHE_ERR_TIMEOUT.  The only device-to-host read in the library apart from
+ * Synchronises the stream, reads the workspace's status word and returns 0,
+ * AIRCACHE_ERR_TIMEOUT (a bounded wait gave up) or AIRCACHE_ERR_INCONSISTENT
+ * (aircache_compact met values that do not fit the buffers).  The only
+ * device-to-host read in the library apart from
  * aircache_pipeline_host().
  */
 int aircache_check_status(void *workspace, int64_t workspace_bytes, void *cuda_stream);

@@ -24,6 +24,7 @@ ERR_CAPACITY = -5
 ERR_CUDA = -6
 ERR_TIMEOUT = -7
 ERR_STATIC_SCRATCH = -8
+ERR_INCONSISTENT = -9
 
 
 class AirCacheError(RuntimeError):

@@ -147,6 +147,8 @@ const char *aircache_strerror(int code) {
         case AIRCACHE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case AIRCACHE_ERR_STATIC_SCRATCH:
             return "problem needs more scratch than the built-in array of aircache_decode_attn_static holds";
+        case AIRCACHE_ERR_INCONSISTENT:
+            return "budgets, offsets or kept lists on the device do not fit the buffers; the rows concerned were not written";
         default: return "unknown error code";
     }
 }
@@ -293,6 +295,7 @@ int aircache_check_status(void *workspace, int64_t workspace_bytes, void *cuda_s
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost,
                                       (cudaStream_t)cuda_stream));
     AIRCACHE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    if (word == kStatusInconsistent) return AIRCACHE_ERR_INCONSISTENT;
     return word ? AIRCACHE_ERR_TIMEOUT : AIRCACHE_OK;
 }
 

@@ -15,6 +15,9 @@ constexpr int kMaxRegions = 1792;     // L * B (the decode kernel keeps the unit
 constexpr int kMaxDecodeCtas = 256;   // upper bound on the persistent decode grid (sizes the partial slots)
 constexpr int kScoreKeyTile = 128;    // visual keys per CTA of the importance pass
 constexpr float kLog2e = 1.4426950408889634f;
+// status word left by aircache_compact when the device-side budgets / offsets / lists do not fit the buffers
+// (waits that gave up leave small numbers that say which wait)
+constexpr uint32_t kStatusInconsistent = 100;
 constexpr int64_t kStatusBytes = 256 + (int64_t)kMaxRegions * 4;  // status word + tickets, at the start of the workspace
 // Decode launches over few regions plan per warp, in registers (head-split launches: at least two KV heads per
 // region, so at most kMaxDecodeCtas / 2 regions; by-region launches: up to 64 regions), and keep, per CTA, the

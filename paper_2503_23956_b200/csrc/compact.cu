@@ -57,7 +57,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
                                                              const int32_t *__restrict__ budgets,
                                                              const int64_t *__restrict__ offsets, int n_visual,
                                                              int n_text, int slack, int64_t first_row,
-                                                             int32_t *__restrict__ kept) {
+                                                             int32_t *__restrict__ kept, int64_t kept_cap,
+                                                             uint32_t *status) {
     extern __shared__ uint32_t s_keys[];
     __shared__ int s_hist[256];
     __shared__ int s_warp[kSelThreads / 32];
@@ -68,7 +69,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float *__rest
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int r = blockIdx.x;
     const int k = budgets[r];
-    int32_t *out = kept + (offsets[r] - first_row - (int64_t)r * (n_text + slack));
+    // the region's list starts after the kept rows of the regions before it; budgets and offsets come from
+    // device memory, so a pair that does not fit the list buffer is reported instead of followed
+    const int64_t start = offsets[r] - first_row - (int64_t)r * (n_text + slack);
+    if (k < 0 || k > n_visual || start < 0 || start + k > kept_cap) {
+        if (threadIdx.x == 0) atomicExch(status, kStatusInconsistent);
+        return;
+    }
+    int32_t *out = kept + start;
     const float *x = scores + (int64_t)r * n_visual;
     if (k <= 0) return;
     if (k >= n_visual) {
@@ -168,6 +176,9 @@ struct GatherParams {
     const int32_t *budgets;
     const int32_t *kept;
     int64_t rows_cap;  // rows covered by the launch
+    int64_t total_rows;  // rows the output buffers hold
+    int64_t kept_cap;    // entries the kept-list buffer holds
+    uint32_t *status;
     int64_t first_row; // rows of the shared buffers in front of this cache's first region
     int L, B, Hkv, d, Nv, Nt, slack;
     int Hc;   // cells per (layer, sequence): 1, or the KV heads in per-KV-head mode (a row then holds one head)
@@ -230,7 +241,9 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
             if (idx >= n_text_rows) continue;
             const int r = idx / p.Nt, j = idx - r * p.Nt;
             src_off[i] = src_of(r, p.Nv + j);
-            dst_row[i] = p.offsets[r] + p.budgets[r] + j;
+            const int64_t dst = p.offsets[r] + p.budgets[r] + j;
+            if (dst < 0 || dst >= p.total_rows) atomicExch(p.status, kStatusInconsistent);   // not written
+            else dst_row[i] = dst;
         }
         copy_rows(src_off, dst_row);
     }
@@ -238,7 +251,11 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
     // ---- kept visual rows, once the selection has written its lists ----
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t per = p.Nt + p.slack;   // offsets[r] - first_row - r * per = kept rows of the regions before r
-    const int64_t n_kept = p.offsets[n_regions] - p.first_row - (int64_t)n_regions * per;
+    int64_t n_kept = p.offsets[n_regions] - p.first_row - (int64_t)n_regions * per;
+    if (n_kept < 0 || n_kept > p.kept_cap) {
+        if (threadIdx.x == 0) atomicExch(p.status, kStatusInconsistent);
+        n_kept = 0;
+    }
     for (int64_t first = warp0 * kGatherRowsPerWarp; first < n_kept; first += row_step) {
         int64_t src_off[kGatherRowsPerWarp], dst_row[kGatherRowsPerWarp];
 #pragma unroll
@@ -256,8 +273,14 @@ __global__ void __launch_bounds__(kGatherThreads, 4) gather_kernel(GatherParams 
             const int r = lo;
             const int64_t base = p.offsets[r];
             const int j = (int)(idx - (base - p.first_row - (int64_t)r * per));
-            src_off[i] = src_of(r, p.kept[idx]);
-            dst_row[i] = base + j;
+            const int tok = p.kept[idx];
+            const int64_t dst = base + j;
+            if (tok < 0 || tok >= p.Nv || dst < 0 || dst >= p.total_rows) {
+                atomicExch(p.status, kStatusInconsistent);   // not copied
+            } else {
+                src_off[i] = src_of(r, tok);
+                dst_row[i] = dst;
+            }
         }
         copy_rows(src_off, dst_row);
     }
@@ -284,15 +307,17 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     const WsLayout w = ws_layout(s);
     const int LB = (int)n_cells(s);
     int32_t *kept = kept_idx ? kept_idx : ws_ptr<int32_t>(ws, w.kept);
+    uint32_t *status = ws_ptr<uint32_t>(ws, w.status);
+    const int64_t kept_cap = (int64_t)s->batch * kept_per_sequence(s, ratio);
     if (s->n_visual <= kSelSmemKeys) {
         const size_t smem = (size_t)s->n_visual * 4;
         AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                kSelSmemKeys * 4));
         select_kernel<true><<<LB, kSelThreads, smem, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
-                                                           s->slack, out->first_row, kept);
+                                                           s->slack, out->first_row, kept, kept_cap, status);
     } else {
         select_kernel<false><<<LB, kSelThreads, 0, st>>>(scores, budgets, out->offsets, s->n_visual, s->n_text,
-                                                         s->slack, out->first_row, kept);
+                                                         s->slack, out->first_row, kept, kept_cap, status);
     }
     AIRCACHE_LAUNCH_CHECK();
 
@@ -302,7 +327,10 @@ int launch_compact(const aircache_shape_t *s, const aircache_full_t *f, const fl
     p.k_out = (uint16_t *)out->k; p.v_out = (uint16_t *)out->v;
     p.offsets = out->offsets; p.lens = out->lens; p.budgets = budgets; p.kept = kept;
     p.first_row = out->first_row;
-    p.rows_cap = (int64_t)s->batch * kept_per_sequence(s, ratio) + (int64_t)LB * (s->n_text + s->slack);
+    p.rows_cap = kept_cap + (int64_t)LB * (s->n_text + s->slack);
+    p.total_rows = out->total_rows;
+    p.kept_cap = kept_cap;
+    p.status = status;
     p.Hc = cells_of(s);
     p.L = s->n_layers; p.B = s->batch; p.Hkv = s->n_kv_heads; p.d = s->head_dim;
     p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack;

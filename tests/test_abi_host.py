@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(handle, n), f"{n} declared in aircache.h but not exported"
     assert sorted(ac.exported_symbols()) == names, "binding and header disagree"
-    assert ac.aircache_version() == 101
+    assert ac.aircache_version() == 102
 
 
 def test_strerror_covers_all_codes():

@@ -811,6 +811,43 @@ def test_bounded_wait_ends_in_an_error_code_not_a_hang():
     assert gp.status() == 0 and torch.isfinite(gp.out).all()
 
 
+@pytest.mark.parametrize("damage", ["budgets_too_large", "offsets_beyond_the_buffers", "offsets_negative"])
+def test_compaction_reports_budgets_and_offsets_that_do_not_fit(oracle, damage):
+    """aircache_compact reads budgets and offsets from device memory.  When a caller has written values there
+    that do not fit the buffers, the rows and list entries concerned are left unwritten, nothing outside the
+    buffers is touched (guard rows behind K', V' and the kept list stay as they were), aircache_check_status
+    reports AIRCACHE_ERR_INCONSISTENT, and after a reset the same buffers serve a correct run."""
+    import paper_2503_23956_b200 as ac
+    wl = CASES["s7b"]
+    ref = oracle_path(oracle, wl)
+    gp = make_gpu(wl, ref)
+    guard = 64
+    gp.k_c = torch.full((gp.rows + guard,) + tuple(gp.k_c.shape[1:]), 1.5, dtype=torch.bfloat16, device=DEV)
+    gp.v_c = torch.full_like(gp.k_c, 2.5)
+    gp.kept = torch.full((gp.kept_n + guard,), -7, dtype=torch.int32, device=DEV)
+    gp.cache = ac.ragged_view(gp.k_c, gp.v_c, gp.offsets, gp.lens, gp.rows)
+    gp.score(ref["qw"].to(DEV))
+    gp.budget()
+    assert gp.status() == 0
+    if damage == "budgets_too_large":
+        gp.budgets.fill_(wl.n_visual)
+    elif damage == "offsets_beyond_the_buffers":
+        gp.offsets[1:] += 1 << 40
+    else:
+        gp.offsets[1:] -= 1 << 40
+    gp.compact()
+    assert gp.status() == ac.ERR_INCONSISTENT
+    assert ac.aircache_strerror(ac.ERR_INCONSISTENT) != ac.aircache_strerror(-12345)
+    assert (gp.k_c[gp.rows:] == 1.5).all() and (gp.v_c[gp.rows:] == 2.5).all()
+    assert (gp.kept[gp.kept_n:] == -7).all()
+    ac.aircache_reset_status(gp.ws)
+    gp.budget()
+    gp.compact()
+    assert gp.status() == 0
+    compare_cache(gp, ref["compact"])
+    assert (gp.k_c[gp.rows:] == 1.5).all() and (gp.kept[gp.kept_n:] == -7).all()
+
+
 @pytest.mark.parametrize("pinned_v", [True, False])
 def test_pipeline_host_matches_staged_calls(oracle, pinned_v):
     """Host inputs in, host outputs out, equal to the staged calls bit for bit - with V in page-locked memory
