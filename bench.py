@@ -562,10 +562,10 @@ def run_cuda(args):
     }
     if rank == 0 and not args.no_e2e:
         result["e2e"] = run_e2e(ac, wl, sh, reqs[0], n_dec, dev, min(args.steps, 3))
-    if rank == 0 and world == 1 and args.extra not in ("", "none"):
-        result["allocation_ablation"] = allocation_ablation(ac, wl, reqs[0])
     del reqs
     torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and args.extra not in ("", "none"):
+        result["allocation_ablation"] = allocation_ablation(ac, dev)
 
     # every other configuration and sweep point, briefly
     if rank == 0 and world == 1 and args.extra not in ("", "none"):
@@ -626,20 +626,29 @@ def dense_window_score(wl, s, reps=10):
             "note": "both passes of Eq. 7 on tcgen05; FLOPs count the unpadded rows, keys are read once per pass"}
 
 
-def allocation_ablation(ac, wl, s):
+def allocation_ablation(ac, dev, spec="c2", text_amp_hi=8.0):
     """The allocation variants of the paper's ablation (strength + skewness, strength only, skewness only,
-    uniform) as budget vectors over the layers of sequence 0, from aircache_budget's mode flag on the scores of
-    one resident request, and the Jensen-Shannon divergence (bits) of every variant's distribution of the budget
-    over the layers from the combined rule's."""
-    s.score(s.qw)
+    uniform) as budget vectors over the layers of sequence 0, from aircache_budget's mode flag, and the
+    Jensen-Shannon divergence (bits) of every variant's distribution of the budget over the layers from the
+    combined rule's.  Run on a variant of the workload whose candidate-window text keys take a share of the
+    softmax that differs by layer (generator option text_amp_hi): on the plain configurations the visual tokens
+    hold nearly all of the mass in every layer and the strength term has nothing to tell apart."""
+    from paper_2503_23956_b200.session import Session
+    from workloads import full_cache, window_queries
+    wl = pick_workload(spec, None).with_(text_amp_hi=text_amp_hi)
+    s = Session(shape_of(ac, wl), wl.ratio, wl.alpha, dev)
+    k = full_cache(wl, "k", dev)
+    s.set_full(logical(k), logical(k))
+    s.score(window_queries(wl, dev))
     LB = wl.n_layers * wl.batch
     budgets = torch.empty_like(s.budgets)
+    strength = torch.empty_like(s.strength)
     layout = ac.ragged_view(None, None, torch.empty(LB + 1, dtype=torch.int64, device=s.dev),
                             torch.empty(LB, dtype=torch.int32, device=s.dev), 0)
     names = ["strength_and_skewness", "strength_only", "skewness_only", "uniform"]
     vec = {}
     for mode, name in enumerate(names):
-        ac.aircache_budget(s.sh, s.scores, s.ratio, mode, budgets, None, None, layout, s.ws)
+        ac.aircache_budget(s.sh, s.scores, s.ratio, mode, budgets, strength, None, layout, s.ws)
         vec[name] = budgets[:, 0].cpu().numpy().astype(np.float64)
 
     def js(a, b):
@@ -652,7 +661,10 @@ def allocation_ablation(ac, wl, s):
         return 0.5 * kl(pa, m) + 0.5 * kl(pb, m)
 
     ref = vec[names[0]]
-    return {"budgets_per_layer_sequence0": {n: [int(x) for x in v] for n, v in vec.items()},
+    st = strength[:, 0].cpu().numpy()
+    return {"workload": describe(wl) + f" text_amp_hi={text_amp_hi:g}",
+            "strength_per_layer_sequence0": [round(float(x), 4) for x in st],
+            "budgets_per_layer_sequence0": {n: [int(x) for x in v] for n, v in vec.items()},
             "js_divergence_bits_vs_combined": {n: js(vec[n], ref) for n in names[1:]}}
 
 

@@ -32,6 +32,9 @@ CASES = {
     # the paper's own window: every text token a candidate (W = N_t = 128: two mask words per head)
     "w128": small("w128", L=2, Hq=28, Hkv=4, d=128, B=1, Nv=700, Nt=128, W=128),
     "w100": small("w100", L=1, Hq=8, Hkv=2, d=64, B=2, Nv=300, Nt=100, W=100),
+    # the window's text keys take a share of the softmax that differs by layer: the strength term of Eq. 11 moves
+    # the budgets (on the other cases the visual tokens hold nearly all of the mass in every layer)
+    "textmass": small("textmass", L=6, B=1, Nv=600, Nt=32, text_amp_hi=8.0),
     # long regions cut across many CTAs with an odd head count (padded partial slots, multi-round merge)
     "kv1long": small("kv1long", L=2, Hq=3, Hkv=1, d=128, B=1, Nv=9000, Nt=9, W=4, ratio=0.9),
     # more (region, KV head) pairs than SMs: the by-region decode schedule with several regions per CTA

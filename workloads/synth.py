@@ -8,6 +8,9 @@ Recipe (per layer l, sequence b, KV head g):
     a_lb ~ U(0.5, 4) differs per layer (so the skewness of the importance scores differs per
     layer) and q_gain = sqrt(head_dim).  For video-shaped workloads the planted tokens are
     drawn only from a few "hot" frames chosen per sequence.
+  * Optional (text_amp_hi > 0, off in the five configurations): the text keys of the candidate window get
+    += t_lb * u_lbg with t_lb ~ U(0, text_amp_hi) per layer, so that the window's own text keys take a share
+    of the softmax that differs by layer (and with it the allocation strength of the layers).
   * Small random objects (a_lb, u_lbg, planted sets, hot frames) come from numpy's PCG64
     seeded with (seed, sequence, tag); they are computed on the host and uploaded.
 All fp32 arithmetic on the large tensors is one addition of two fp32 numbers followed by a
@@ -46,6 +49,7 @@ class Workload:
     amp_hi: float = 4.0
     n_frames: int = 0             # > 0: video-shaped, n_visual = n_frames * tokens per frame
     hot_frames: int = 3
+    text_amp_hi: float = 0.0      # > 0: the text keys of the candidate window get + t_lb * u_lbg, t_lb ~ U(0, text_amp_hi)
     seed: int = BASE_SEED
 
     @property
@@ -153,6 +157,7 @@ class Plan:
     u: np.ndarray            # f32 [L, B, Hkv, d]    unit directions
     planted: np.ndarray      # bool [L, B, Nv]       planted visual tokens
     hot: np.ndarray | None   # i64 [B, hot_frames]   hot frames (video-shaped only)
+    text_amp: np.ndarray | None = None   # f32 [L, B]  amplitude t_lb on the window's text keys (text_amp_hi > 0 only)
 
 
 _PLANS: dict = {}
@@ -181,7 +186,13 @@ def plan(wl: Workload) -> Plan:
         g = _rng(wl, b, "plant")
         for l in range(L):
             planted[l, b, g.choice(pool, n_plant, replace=False)] = True
-    p = Plan(amp, u, planted, hot)
+    text_amp = None
+    if wl.text_amp_hi > 0:
+        # the window's text keys pull attention mass away from the visual tokens, by a different amount in every
+        # layer: the visual share of the softmax (the allocation strength of Eq. 9) then differs by layer
+        text_amp = np.stack([_rng(wl, b, "textamp").uniform(0.0, wl.text_amp_hi, size=L) for b in range(B)],
+                            axis=1).astype(np.float32)
+    p = Plan(amp, u, planted, hot, text_amp)
     _PLANS[wl] = p
     return p
 
@@ -202,6 +213,8 @@ def full_cache(wl: Workload, which: str, device="cpu", layers=None, seqs=None) -
                 mask = torch.from_numpy(pl.planted[l, b]).to(device)                     # bool [Nv]
                 zv = z[:Nv]
                 z[:Nv] = torch.where(mask[:, None, None], zv + add[None], zv)
+                if pl.text_amp is not None:
+                    z[N - wl.window:] += torch.from_numpy(pl.text_amp[l, b] * pl.u[l, b]).to(device)[None]
             out[li, bi] = z.to(torch.bfloat16)
     return out
 
