@@ -1,13 +1,13 @@
 // aircache_budget: strength and skewness of every region's importance distribution (Eq. 9-10), the
 // layer-wise budget of Eq. 11 turned into integer row counts, and the row offsets of the ragged cache.
 //
-// One launch.  Every CTA reduces one region (three fp64 block reductions over the fp32 scores, which it
+// One launch.  Every CTA reduces one cell (three fp64 block reductions over the fp32 scores, which it
 // keeps in registers: sum; squared deviations; cubed standardised deviations; fixed reduction tree).  The
-// CTA that finishes last (a ticket in the workspace, put back to zero for the next call) then runs the
-// allocation for all sequences: one warp per sequence, sums over the layers taken by one lane in layer
-// order and every fp64 operation individually rounded (no fused multiply-add), so that the integer
-// budgets are the ones the sequential definition gives; divisions, floors and the ranking of the
-// fractional parts run across the lanes.  Finally the same CTA scans the region sizes into offsets.
+// CTA that finishes a SEQUENCE last (one ticket per sequence in the workspace, put back to zero for the next
+// call) runs that sequence's allocation with one warp: sums over the cells taken by one lane in cell order
+// and every fp64 operation individually rounded (no fused multiply-add), so that the integer budgets are
+// the ones the sequential definition gives; divisions, floors and the ranking of the fractional parts run
+// across the lanes.  The CTA that finishes the last sequence scans the region sizes into offsets.
 #include <math.h>
 
 #include "common.cuh"
@@ -25,7 +25,8 @@ struct BudgetParams {
     int32_t *budgets;        // [L,B]
     int64_t *offsets;        // [L*B+1]
     int32_t *lens;           // [L*B]
-    uint32_t *ticket;        // zero between calls
+    uint32_t *ticket;        // sequences allocated so far; zero between calls
+    uint32_t *seq_ticket;    // [B] cells of the sequence reduced so far; zero between calls
     int L, B, Hc, Nv, Nt, slack, mode;   // Hc: cells per (layer, sequence) - the KV heads in per-KV-head mode, else 1
     long long total_kept;    // T per sequence
     long long first_row;     // rows of the shared buffers in front of this cache's first region
@@ -48,21 +49,18 @@ __device__ __forceinline__ double warp_bcast(double v, int src) {
     return __shfl_sync(0xffffffffu, v, src);
 }
 
-// Eq. 11 and the integer budgets of sequence b, by one warp.  st/sk/w/share are arrays over all cells in shared
-// memory; the sequence's cells - its layers, or its (layer, KV head) pairs in per-KV-head mode, layer-major -
-// are numbered l = 0 .. L*Hc - 1 here and sit at AT(l); act flags cells that still take part in the
-// proportional split.
-__device__ void allocate_sequence(const BudgetParams &p, int b, const double *st, const double *sk, double *w,
+// Eq. 11 and the integer budgets of one sequence, by one warp.  st/sk/w/share/bud/act are arrays in shared memory
+// over the sequence's cells - its layers, or its (layer, KV head) pairs in per-KV-head mode, layer-major -
+// numbered l = 0 .. n - 1; act flags cells that still take part in the proportional split.
+__device__ void allocate_sequence(const BudgetParams &p, int n, const double *st, const double *sk, double *w,
                                   double *share, unsigned char *act, int *bud) {
-    const int L = p.L * p.Hc, lane = threadIdx.x & 31;
-    const int B = p.B, Hc = p.Hc;
-#define AT(l) ((((l) / Hc) * B + b) * Hc + (l) % Hc)
+    const int L = n, lane = threadIdx.x & 31;
     // across-layer means: one lane, layer order (this fixes the rounding of the sums)
     double mean_t = 0.0, mean_k = 0.0;
     if (lane == 0) {
         for (int l = 0; l < L; ++l) {
-            mean_t = __dadd_rn(mean_t, st[AT(l)]);
-            const double s = sk[AT(l)];
+            mean_t = __dadd_rn(mean_t, st[l]);
+            const double s = sk[l];
             mean_k = __dadd_rn(mean_k, s > 0.0 ? s : 0.0);
         }
         mean_t = __ddiv_rn(mean_t, (double)L);
@@ -71,8 +69,8 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     mean_t = warp_bcast(mean_t, 0);
     mean_k = warp_bcast(mean_k, 0);
     for (int l = lane; l < L; l += 32) {
-        const double t = st[AT(l)];
-        double s = sk[AT(l)];
+        const double t = st[l];
+        double s = sk[l];
         if (s < 0.0) s = 0.0;
         const double nt = mean_t > 0.0 ? __ddiv_rn(t, mean_t) : 1.0;
         const double nk = mean_k > 0.0 ? __ddiv_rn(s, mean_k) : 1.0;
@@ -81,8 +79,8 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
         else if (p.mode == 1) ww = nt;
         else if (p.mode == 2) ww = nk;
         else ww = 1.0;
-        w[AT(l)] = ww;
-        act[AT(l)] = 1;
+        w[l] = ww;
+        act[l] = 1;
     }
     __syncwarp();
     long long R = p.total_kept;
@@ -92,20 +90,20 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
         int n_active = 0;
         if (lane == 0) {
             for (int l = 0; l < L; ++l)
-                if (act[AT(l)]) { wsum = __dadd_rn(wsum, w[AT(l)]); ++n_active; }
+                if (act[l]) { wsum = __dadd_rn(wsum, w[l]); ++n_active; }
         }
         wsum = warp_bcast(wsum, 0);
         n_active = __shfl_sync(0xffffffffu, n_active, 0);
         if (n_active == 0) break;
         int moved = 0;
         for (int l = lane; l < L; l += 32) {
-            if (!act[AT(l)]) continue;
-            const double sh = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, w[AT(l)]), wsum)
+            if (!act[l]) continue;
+            const double sh = wsum > 0.0 ? __ddiv_rn(__dmul_rn((double)R, w[l]), wsum)
                                          : __ddiv_rn((double)R, (double)n_active);
-            share[AT(l)] = sh;
+            share[l] = sh;
             if (sh >= (double)p.Nv) {
-                bud[AT(l)] = p.Nv;
-                act[AT(l)] = 0;
+                bud[l] = p.Nv;
+                act[l] = 0;
                 ++moved;
             }
         }
@@ -118,12 +116,12 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     // floors, then the largest fractional parts (ties to the lower layer) take one more row each
     int given = 0;
     for (int l = lane; l < L; l += 32) {
-        if (!act[AT(l)]) continue;
-        const double sh = share[AT(l)];
+        if (!act[l]) continue;
+        const double sh = share[l];
         const int f = (int)floor(sh);
-        bud[AT(l)] = f;
+        bud[l] = f;
         given += f;
-        share[AT(l)] = __dsub_rn(sh, (double)f);
+        share[l] = __dsub_rn(sh, (double)f);
     }
     long long given_all = given;
 #pragma unroll
@@ -133,21 +131,20 @@ __device__ void allocate_sequence(const BudgetParams &p, int b, const double *st
     // a layer gets the extra row iff fewer than `left` active layers precede it in the order
     // (fraction descending, layer ascending): the same set the one-at-a-time selection picks
     for (int l = lane; l < L; l += 32) {
-        if (!act[AT(l)]) continue;
-        const double fr = share[AT(l)];
+        if (!act[l]) continue;
+        const double fr = share[l];
         long long rank = 0;
         for (int l2 = 0; l2 < L; ++l2) {
-            if (!act[AT(l2)]) continue;
-            const double f2 = share[AT(l2)];
+            if (!act[l2]) continue;
+            const double f2 = share[l2];
             rank += (f2 > fr) || (f2 == fr && l2 < l);
         }
-        if (rank < left) bud[AT(l)] += 1;
+        if (rank < left) bud[l] += 1;
     }
     __syncwarp();
 }
-#undef AT
 
-__global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
+__global__ void __launch_bounds__(kThreads, 2) budget_kernel(BudgetParams p) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ double s_part[kThreads / 32];
     __shared__ int s_is_last;
@@ -206,35 +203,54 @@ __global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
             p.strength[blockIdx.x] = s;
             p.skewness[blockIdx.x] = sigma > 0.0 ? __dmul_rn(pre, cube) : 0.0;
             __threadfence();
-            const unsigned t = atomicAdd(p.ticket, 1u);
-            s_is_last = (t == (unsigned)LB - 1);
-            if (s_is_last) { *p.ticket = 0; __threadfence(); }
+            // cell index = (l * B + b) * Hc + g: the sequence is the middle coordinate
+            const int b = (blockIdx.x / p.Hc) % p.B;
+            const unsigned t = atomicAdd(p.seq_ticket + b, 1u);
+            s_is_last = (t == (unsigned)(p.L * p.Hc) - 1);
+            if (s_is_last) { p.seq_ticket[b] = 0; __threadfence(); }
         }
         __syncthreads();
         if (!s_is_last) return;
     }
 
-    // ---------------- the last CTA: allocation for every sequence, then the offsets ----------------
+    // ---------------- the sequence's last CTA: its allocation ----------------
+    const int b = (blockIdx.x / p.Hc) % p.B;
+    const int n = p.L * p.Hc;   // cells of the sequence
     double *st = reinterpret_cast<double *>(s_dyn);
-    double *sk = st + LB;
-    double *w = sk + LB;
-    double *share = w + LB;
-    int *bud = reinterpret_cast<int *>(share + LB);
-    unsigned char *act = reinterpret_cast<unsigned char *>(bud + LB);
-    for (int i = tid; i < LB; i += kThreads) {
-        st[i] = __ldcg(p.strength + i);
-        sk[i] = __ldcg(p.skewness + i);
+    double *sk = st + n;
+    double *w = sk + n;
+    double *share = w + n;
+    int *bud = reinterpret_cast<int *>(share + n);
+    unsigned char *act = reinterpret_cast<unsigned char *>(bud + n);
+    // cell l of the sequence sits at ((l / Hc) * B + b) * Hc + l % Hc
+    auto at = [&](int l) { return ((l / p.Hc) * p.B + b) * p.Hc + l % p.Hc; };
+    for (int l = tid; l < n; l += kThreads) {
+        st[l] = __ldcg(p.strength + at(l));
+        sk[l] = __ldcg(p.skewness + at(l));
     }
     __syncthreads();
-    for (int b = tid >> 5; b < p.B; b += kThreads / 32) allocate_sequence(p, b, st, sk, w, share, act, bud);
+    if (tid < 32) allocate_sequence(p, n, st, sk, w, share, act, bud);
     __syncthreads();
+    for (int l = tid; l < n; l += kThreads) {
+        __stcg(p.budgets + at(l), bud[l]);
+        p.lens[at(l)] = bud[l] + p.Nt;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned t = atomicAdd(p.ticket, 1u);
+        s_is_last = (t == (unsigned)p.B - 1);
+        if (s_is_last) { *p.ticket = 0; __threadfence(); }
+    }
+    __syncthreads();
+    if (!s_is_last) return;
 
-    // offsets: exclusive scan of (budget + Nt + slack) over r = l*B + b
+    // ---------------- the last sequence's CTA: offsets = exclusive scan of (budget + Nt + slack) over the cells ----
     __shared__ long long s_warp[kThreads / 32];
     const int per = (LB + kThreads - 1) / kThreads;
     const int i0 = min(LB, tid * per), i1 = min(LB, i0 + per);
     long long local = 0;
-    for (int i = i0; i < i1; ++i) local += bud[i] + p.Nt + p.slack;
+    for (int i = i0; i < i1; ++i) local += __ldcg(p.budgets + i) + p.Nt + p.slack;
     long long incl = local;
     const int lane = tid & 31, warp = tid >> 5;
 #pragma unroll
@@ -257,9 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) budget_kernel(BudgetParams p) {
     long long run = p.first_row + incl - local + (warp > 0 ? s_warp[warp - 1] : 0);
     for (int i = i0; i < i1; ++i) {
         p.offsets[i] = run;
-        p.lens[i] = bud[i] + p.Nt;
-        p.budgets[i] = bud[i];
-        run += bud[i] + p.Nt + p.slack;
+        run += __ldcg(p.budgets + i) + p.Nt + p.slack;
     }
     if (tid == kThreads - 1) p.offsets[LB] = p.first_row + s_warp[kThreads / 32 - 1];
 }
@@ -278,10 +292,13 @@ int launch_budget(const aircache_shape_t *s, const float *scores, double ratio, 
     p.offsets = layout->offsets;
     p.lens = layout->lens;
     p.ticket = ws_ptr<uint32_t>(ws, w.status) + 2;   // second word pair of the status block
+    // one ticket per sequence: the decode kernel's split-K tickets, which every user leaves at zero (calls that
+    // share a workspace are ordered on one stream)
+    p.seq_ticket = ws_ptr<uint32_t>(ws, w.tickets);
     p.L = s->n_layers; p.B = s->batch; p.Hc = cells_of(s); p.Nv = s->n_visual; p.Nt = s->n_text; p.slack = s->slack; p.mode = mode;
     p.total_kept = kept_per_sequence(s, ratio);
     p.first_row = layout->first_row;
-    const size_t smem = (size_t)LB * (4 * 8 + 4 + 1) + 16;
+    const size_t smem = (size_t)s->n_layers * cells_of(s) * (4 * 8 + 4 + 1) + 16;
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(budget_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     budget_kernel<<<LB, kThreads, smem, st>>>(p);
     AIRCACHE_LAUNCH_CHECK();

@@ -62,8 +62,11 @@ constexpr float kNegBig = -1.0e30f;
 // ---------------------------------------------------------------------------------------------
 // Eq. 4-5 and the elite-row table
 // ---------------------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(128, 6) elite_kernel(ScoreParams p) {
+// QREG: the row's query is held in registers (64 of them at d = 128, two CTAs per SM) - worth it when a thread
+// takes many rows against many text keys, i.e. when every candidate is elite (alpha = 0); otherwise the row is
+// re-read from L1 per text key and six CTAs share an SM.
+template <int D, bool QREG>
+__global__ void __launch_bounds__(128, QREG ? 2 : 6) elite_kernel(ScoreParams p) {
     constexpr int KS = D + 8;   // padded row: 16-byte reads of consecutive rows fall into different banks
     extern __shared__ __align__(16) uint16_t s_dyn[];
     uint16_t *s_k = s_dyn;                 // [W][KS]   candidate keys
@@ -167,14 +170,19 @@ __global__ void __launch_bounds__(128, 6) elite_kernel(ScoreParams p) {
 #pragma unroll 4
             for (int c = 0; c < D / 8; ++c) qb[c] = __ldg(qq + c);
         }
+        uint4 qr[QREG ? D / 8 : 1];
+        if (QREG) {
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) qr[c] = __ldg(qq + c);
+        }
         float m = kNegBig, z = 0.0f;
         for (int w2 = 0; w2 <= w; ++w2) {
             if (!elite(w2)) continue;
             const uint4 *kk = reinterpret_cast<const uint4 *>(s_k + w2 * KS);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 4
+#pragma unroll QREG ? D / 8 : 4
             for (int c = 0; c < D / 8; ++c) {
-                const uint4 a = __ldg(qq + c), bb = kk[c];
+                const uint4 a = QREG ? qr[c] : __ldg(qq + c), bb = kk[c];
                 a0 = fmaf(bf16lo(a.x), bf16lo(bb.x), a0); a1 = fmaf(bf16hi(a.x), bf16hi(bb.x), a1);
                 a2 = fmaf(bf16lo(a.y), bf16lo(bb.y), a2); a3 = fmaf(bf16hi(a.y), bf16hi(bb.y), a3);
                 a0 = fmaf(bf16lo(a.z), bf16lo(bb.z), a0); a1 = fmaf(bf16hi(a.z), bf16hi(bb.z), a1);
@@ -1196,8 +1204,13 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
 
     const int64_t groups = (int64_t)p.n_lb * p.Hkv;
     const size_t elite_smem = (size_t)(p.W + p.G) * (p.d + 8) * 2;
-    if (s->head_dim == 64) elite_kernel<64><<<(unsigned)groups, 128, elite_smem, st>>>(p);
-    else elite_kernel<128><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+    if (p.keep_all) {
+        if (s->head_dim == 64) elite_kernel<64, true><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+        else elite_kernel<128, true><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+    } else {
+        if (s->head_dim == 64) elite_kernel<64, false><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+        else elite_kernel<128, false><<<(unsigned)groups, 128, elite_smem, st>>>(p);
+    }
     AIRCACHE_LAUNCH_CHECK();
     // alpha = 0 keeps all G*W window queries: the dense contraction goes to tcgen05 (if a tensor map over the
     // caller's strides can be made; otherwise the mma.sync passes handle it as well)
