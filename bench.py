@@ -55,7 +55,7 @@ Q_RING, O_RING = 16, 8
 # batch 16, the largest case the capture rules allow; traffic grows in proportion to the rows, so it is scaled
 # to the launch that was timed).  Valid only for the kernel source it was taken on (sha1 of csrc/decode.cu,
 # first 12 hex); null otherwise.
-NCU_TRAFFIC = {"workload": "c3", "decode_cu_sha1": "", "bytes_per_valid_row": None}
+NCU_TRAFFIC = {"workload": "c3", "decode_cu_sha1": "275867bb0ec6", "bytes_per_valid_row": 2101.25}
 
 
 def parse_args():
