@@ -846,15 +846,70 @@ __device__ __forceinline__ void load_key_tile(uint32_t dst, const CUtensorMap *t
         tma_load_5d(dst + sub * DenseCfg<D>::SUB_BYTES, tm, sub * 64, c[1], c[2], c[3], c[4], bar);
 }
 
-// Pass one, dense.  grid = (chunks, L*B*Hkv), 128 threads.
+// Both dense kernels are warp-specialised: warps 0-3 own one accumulator row per thread (a tensor-memory lane)
+// and run the exponent arithmetic; one thread of warp 4 drives the copies and the tensor core.  Key tiles cycle
+// through NST shared-memory stages (full: TMA landed; empty: the MMAs that read the stage have completed, by
+// tcgen05.commit), accumulators through two halves of 256 tensor-memory columns (acc_full by tcgen05.commit,
+// acc_empty by one arrival per epilogue warp): the MMAs of tile t+1 run while tile t's logits are read back
+// and exponentiated.  Parities follow from running tile counts.  Every wait is bounded.
+constexpr int kDenseThreads = 160;
+
 template <int D>
-__global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+struct DensePipe {
+    using C = DenseCfg<D>;
+    uint32_t full[C::NST], empty[C::NST], acc_full[2], acc_empty[2];   // shared-memory addresses of the mbarriers
+    __device__ void init(uint64_t *s_bar) {
+        for (int i = 0; i < C::NST; ++i) { full[i] = smem_u32(&s_bar[i]); empty[i] = smem_u32(&s_bar[C::NST + i]); }
+        for (int a = 0; a < 2; ++a) { acc_full[a] = smem_u32(&s_bar[2 * C::NST + a]); acc_empty[a] = smem_u32(&s_bar[2 * C::NST + 2 + a]); }
+    }
+    __device__ void init_barriers() const {
+        for (int i = 0; i < C::NST; ++i) { mbar_init(full[i], 1); mbar_init(empty[i], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full[a], 1); mbar_init(acc_empty[a], 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+};
+
+// The driver thread's part for n_tiles key tiles starting at key0: `base` tiles went through the pipe before.
+// a_is_query: the query block is the MMA's A operand (rows on M, pass one), else the key tile is (keys on M).
+template <int D, bool A_IS_QUERY>
+__device__ __forceinline__ bool dense_drive(const DensePipe<D> &pp, const CUtensorMap *tm, const ScoreParams &p,
+                                            uint32_t tmem, uint8_t *s_k, uint8_t *s_q, uint32_t base, int n_tiles,
+                                            int key0, int g, int b, int l, volatile int *s_abort, uint32_t code) {
+    using C = DenseCfg<D>;
+    bool ok = true;
+    int loaded = 0;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+        while (ok && loaded < n_tiles && loaded < t + C::NST) {
+            const uint32_t il = base + loaded, ls = il % C::NST;
+            ok = mbar_wait(pp.empty[ls], ((il / C::NST) & 1) ^ 1, s_abort, p.status, code);
+            if (ok) {
+                load_key_tile<D>(smem_u32(s_k + ls * C::TILE_BYTES), tm, p, key0 + loaded * 128, g, b, l, pp.full[ls]);
+                ++loaded;
+            }
+        }
+        if (!ok) break;
+        const uint32_t it = base + t, st = it % C::NST, a = it & 1;
+        ok = mbar_wait(pp.full[st], (it / C::NST) & 1, s_abort, p.status, code) &&
+             mbar_wait(pp.acc_empty[a], ((it >> 1) & 1) ^ 1, s_abort, p.status, code + 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t k_tile = smem_u32(s_k + st * C::TILE_BYTES), q_blk = smem_u32(s_q);
+        issue_tile_mma<D>(tmem + a * 128, A_IS_QUERY ? q_blk : k_tile, A_IS_QUERY ? k_tile : q_blk);
+        umma_commit(pp.empty[st]);      // the stage may be refilled
+        umma_commit(pp.acc_full[a]);    // the accumulator may be read
+    }
+    return ok;
+}
+
+// Pass one, dense.  grid = (chunks, L*B*Hkv), 160 threads.
+template <int D>
+__global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     using C = DenseCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *s_k = smem;                             // NST key tiles
     uint8_t *s_q = smem + C::NST * C::TILE_BYTES;    // one query block
-    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES);   // full[NST], done
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES);
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort, s_is_last;
 
@@ -868,78 +923,95 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
     const int n_rows = p.row_count[grp];
     float2 *out = p.chunk_stats + ((int64_t)(grp - p.lb0 * p.Hkv) * p.chunks + chunk) * p.cap;
 
+    DensePipe<D> pp;
+    pp.init(s_bar);
     if (tid == 0) {
-        for (int i = 0; i <= C::NST; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pp.init_barriers();
         s_abort = 0;
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 128);
+    if (warp == 4) tmem_alloc(smem_u32(&s_tmem), 256);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t done_bar = smem_u32(&s_bar[C::NST]);
-    uint32_t n_loaded = 0, n_done = 0;   // running counts: they give stage and mbarrier parity
-    bool ok = true;
+    uint32_t base = 0;   // tiles that went through the pipe in earlier row blocks
 
-    for (int row0 = 0; row0 < n_rows && ok; row0 += 128) {
+    for (int row0 = 0; row0 < n_rows; row0 += 128) {
+        __syncthreads();   // the previous block's MMAs have completed (their logits were read): the query block is free
+        if (s_abort) break;
+        if (tid < 128) stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
         __syncthreads();
-        stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
-        __syncthreads();
-        float m = kNegBig, z = 0.f;
-        const uint32_t first = n_loaded;
-        if (tid == 0)
-            for (int i = 0; i < min(C::NST, n_tiles); ++i, ++n_loaded)
-                load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p, key0 + i * 128, g, b, l,
-                                 smem_u32(&s_bar[n_loaded % C::NST]));
-        for (int t = 0; t < n_tiles; ++t) {
-            const uint32_t it = first + t, st = it % C::NST;
-            if (tid == 0) {
-                ok = mbar_wait(smem_u32(&s_bar[st]), (it / C::NST) & 1, &s_abort, p.status, 4);
-                if (ok) {
-                    tc_fence_after();
-                    // rows on M: acc[row][key] = Q_blk * K_tile^T
-                    issue_tile_mma<D>(tmem, smem_u32(s_q), smem_u32(s_k + st * C::TILE_BYTES));
-                    umma_commit(done_bar);
-                }
-            }
-            ok = mbar_wait(done_bar, n_done & 1, &s_abort, p.status, 5);
-            ++n_done;
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll 1
-            for (int cc = 0; cc < 4; ++cc) {
-                float v[32];
-                tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + cc * 32, v);
-                const int kbase = key0 + t * 128 + cc * 32;
-                float mx = kNegBig;
+        if (warp == 4) {
+            if (lane == 0)
+                dense_drive<D, true>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, key0, g, b, l, &s_abort, 4);
+        } else {
+            float m = kNegBig, z = 0.f;
+            bool ok = true;
+            // one chunk of 32 logits of the thread's row: running (max, sum of exp2)
+            auto chunk32 = [&](const uint32_t (&r)[32], int kbase) {
+                float mn, sum = 0.f;
+                if (kbase + 32 <= key1) {
+                    // all 32 keys are real: the scale is positive, so the largest raw logit gives the largest
+                    // scaled one, and the exponent's argument is one fused multiply-add.  Four interleaved
+                    // partial maxima and sums keep the dependent chains short (two warps share a scheduler).
+                    float mx[4], sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    v[j] = kbase + j < key1 ? v[j] * p.sl2 : kNegBig;
-                    mx = fmaxf(mx, v[j]);
-                }
-                const float mn = fmaxf(m, mx);
-                float sum = 0.f;
+                    for (int j = 0; j < 4; ++j) mx[j] = __uint_as_float(r[j]);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) sum += kbase + j < key1 ? fast_exp2(v[j] - mn) : 0.f;
+                    for (int j = 4; j < 32; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(r[j]));
+                    mn = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.sl2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sm[j & 3] += fast_exp2(fmaf(__uint_as_float(r[j]), p.sl2, -mn));
+                    sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
+                } else {
+                    float mx = kNegBig;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (kbase + j < key1) mx = fmaxf(mx, __uint_as_float(r[j]) * p.sl2);
+                    mn = fmaxf(m, mx);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        sum += kbase + j < key1 ? fast_exp2(fmaf(__uint_as_float(r[j]), p.sl2, -mn)) : 0.f;
+                }
                 z = z * fast_exp2(m - mn) + sum;
                 m = mn;
+            };
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t it = base + t, a = it & 1;
+                ok = mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 6);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
+                const int kbase = key0 + t * 128;
+                uint32_t r0[32], r1[32];
+                tmem_ld32_issue(taddr, r0);
+                tmem_ld_wait(r0);
+                tmem_ld32_issue(taddr + 32, r1);
+                chunk32(r0, kbase);
+                tmem_ld_wait(r1);
+                tmem_ld32_issue(taddr + 64, r0);
+                chunk32(r1, kbase + 32);
+                tmem_ld_wait(r0);
+                tmem_ld32_issue(taddr + 96, r1);
+                chunk32(r0, kbase + 64);
+                tmem_ld_wait(r1);
+                // the whole accumulator is in registers: hand it back before the last chunk's arithmetic
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pp.acc_empty[a]);
+                chunk32(r1, kbase + 96);
             }
-            tc_fence_before();
-            __syncthreads();   // the accumulator and the key stage are free again
-            if (tid == 0 && t + C::NST < n_tiles) {
-                load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p,
-                                 key0 + (t + C::NST) * 128, g, b, l, smem_u32(&s_bar[n_loaded % C::NST]));
-                ++n_loaded;
-            }
+            if (ok && row0 + tid < n_rows) __stcg(out + row0 + tid, make_float2(m, z));
         }
-        n_loaded = first + n_tiles;   // every thread tracks the count thread 0 advanced
-        if (ok && row0 + tid < n_rows) __stcg(out + row0 + tid, make_float2(m, z));
+        base += n_tiles;
     }
-    ok = !s_abort;
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 128);
+    const bool ok = !s_abort;
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 256);
+    }
     if (!ok) return;
 
     // last CTA of the group: merge text and chunk statistics (same scheme as stats_kernel)
@@ -950,7 +1022,7 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
         if (s_is_last) __threadfence();
     }
     __syncthreads();
-    if (!s_is_last) return;
+    if (!s_is_last || warp >= 4) return;
     for (int r = warp; r < n_rows; r += 4) {
         float mm = kNegBig, zz = 0.f;
         if (lane == 0) {
@@ -971,11 +1043,9 @@ __global__ void __launch_bounds__(128) dense_stats_kernel(const __grid_constant_
     }
 }
 
-// Pass two, dense.  grid = (ceil(Nv / (128 * KT)), L*B), 128 threads; a CTA owns KT key tiles and thread i the
-// keys 128 * tile + i of them.  Per KV head and block of 128 query rows the block is staged once and the
-// CTA's key tiles stream through a ring of NST stages.
+// Pass two, dense.  grid = (ceil(Nv / (128*KT)), L*B), 160 threads; an epilogue thread owns one key per tile.
 template <int D>
-__global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+__global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     using C = DenseCfg<D>;
     constexpr int KT = C::KT;
     extern __shared__ uint8_t smem_raw[];
@@ -983,88 +1053,96 @@ __global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_cons
     uint8_t *s_k = smem;                             // NST key tiles
     uint8_t *s_q = smem + C::NST * C::TILE_BYTES;    // one query block
     float2 *s_stat = reinterpret_cast<float2 *>(smem + (C::NST + 1) * C::TILE_BYTES);   // (max, weight / normaliser)
-    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES + 128 * 8);   // full[NST], done
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + (C::NST + 1) * C::TILE_BYTES + 128 * 8);
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lb = p.lb0 + blockIdx.y;
     const int l = lb / p.B, b = lb % p.B;
     const int key0 = blockIdx.x * 128 * KT;
     const int n_tiles = min(KT, (p.Nv - key0 + 127) / 128);
 
+    DensePipe<D> pp;
+    pp.init(s_bar);
     if (tid == 0) {
-        for (int i = 0; i <= C::NST; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pp.init_barriers();
         s_abort = 0;
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 0) tmem_alloc(smem_u32(&s_tmem), 128);
+    if (warp == 4) tmem_alloc(smem_u32(&s_tmem), 256);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t done_bar = smem_u32(&s_bar[C::NST]);
-    uint32_t n_loaded = 0, n_done = 0;
-    bool ok = true;
+    uint32_t base = 0;
     float imp[KT];
 #pragma unroll
     for (int t = 0; t < KT; ++t) imp[t] = 0.f;
 
-    for (int g = 0; g < p.Hkv && ok; ++g) {
+    for (int g = 0; g < p.Hkv; ++g) {
         const int grp = lb * p.Hkv + g;
         const int n_rows = p.row_count[grp];
-        for (int row0 = 0; row0 < n_rows && ok; row0 += 128) {
-            const uint32_t first = n_loaded;
-            if (tid == 0)   // the ring is empty here: every tile of the previous block was consumed
-                for (int i = 0; i < min(C::NST, n_tiles); ++i, ++n_loaded)
-                    load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p, key0 + i * 128, g, b,
-                                     l, smem_u32(&s_bar[n_loaded % C::NST]));
-            stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
-            s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
+        for (int row0 = 0; row0 < n_rows; row0 += 128) {
+            __syncthreads();   // the previous block's MMAs have completed: query block and statistics are free
+            if (s_abort) break;
+            if (tid < 128) {
+                stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
+                s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
+            }
             __syncthreads();
-            const int cols = min(128, n_rows - row0);
-#pragma unroll
-            for (int t = 0; t < KT; ++t) {
-                if (t >= n_tiles) break;
-                const uint32_t it = first + t, st = it % C::NST;
-                if (tid == 0) {
-                    ok = mbar_wait(smem_u32(&s_bar[st]), (it / C::NST) & 1, &s_abort, p.status, 6);
-                    if (ok) {
-                        tc_fence_after();
-                        // keys on M: acc[key][row] = K_tile * Q_blk^T
-                        issue_tile_mma<D>(tmem, smem_u32(s_k + st * C::TILE_BYTES), smem_u32(s_q));
-                        umma_commit(done_bar);
-                    }
-                }
-                ok = mbar_wait(done_bar, n_done & 1, &s_abort, p.status, 7);
-                ++n_done;
-                if (!ok) break;
-                tc_fence_after();
-#pragma unroll 1
-                for (int cc = 0; cc < 4; ++cc) {
-                    if (cc * 32 >= cols) break;
-                    float v[32];
-                    tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + cc * 32, v);
-                    float acc = 0.f;
+            if (warp == 4) {
+                if (lane == 0)
+                    dense_drive<D, false>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, key0, g, b, l, &s_abort, 10);
+            } else {
+                const int nch = (min(128, n_rows - row0) + 31) >> 5;   // chunks of 32 rows with a real row in them
+                // 32 rows of the thread's key: probabilities weighted and summed
+                auto chunk32 = [&](const uint32_t (&r)[32], int c0) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};   // interleaved partial sums: short dependent chains
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const float2 sj = s_stat[cc * 32 + j];
-                        acc += fast_exp2(v[j] * p.sl2 - sj.x) * sj.y;
+                        const float2 sj = s_stat[c0 + j];
+                        acc[j & 3] = fmaf(fast_exp2(fmaf(__uint_as_float(r[j]), p.sl2, -sj.x)), sj.y, acc[j & 3]);
+                    }
+                    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+                };
+#pragma unroll
+                for (int t = 0; t < KT; ++t) {
+                    if (t >= n_tiles) break;
+                    const uint32_t it = base + t, a = it & 1;
+                    if (!mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 12)) break;
+                    tc_fence_after();
+                    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
+                    uint32_t r0[32], r1[32];
+                    float acc = 0.f;
+                    tmem_ld32_issue(taddr, r0);
+                    tmem_ld_wait(r0);
+                    if (nch > 1) tmem_ld32_issue(taddr + 32, r1);
+                    acc += chunk32(r0, 0);
+                    if (nch > 1) {
+                        tmem_ld_wait(r1);
+                        if (nch > 2) tmem_ld32_issue(taddr + 64, r0);
+                        acc += chunk32(r1, 32);
+                        if (nch > 2) {
+                            tmem_ld_wait(r0);
+                            if (nch > 3) tmem_ld32_issue(taddr + 96, r1);
+                            acc += chunk32(r0, 64);
+                            if (nch > 3) {
+                                tmem_ld_wait(r1);
+                                acc += chunk32(r1, 96);
+                            }
+                        }
                     }
                     imp[t] += acc;
-                }
-                tc_fence_before();
-                __syncthreads();   // accumulator and key stage are free again
-                if (tid == 0 && t + C::NST < n_tiles) {
-                    load_key_tile<D>(smem_u32(s_k + (n_loaded % C::NST) * C::TILE_BYTES), &tm_k, p,
-                                     key0 + (t + C::NST) * 128, g, b, l, smem_u32(&s_bar[n_loaded % C::NST]));
-                    ++n_loaded;
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pp.acc_empty[a]);
                 }
             }
-            n_loaded = first + n_tiles;
+            base += n_tiles;
         }
-        if (ok && (p.per_head || g == p.Hkv - 1)) {
+        if (s_abort) break;
+        if (tid < 128 && (p.per_head || g == p.Hkv - 1)) {
             // the keys' scores are complete: of this KV group alone, or summed over all of them
             float *out = p.scores + (p.per_head ? (int64_t)grp : (int64_t)lb) * p.Nv;
 #pragma unroll
@@ -1075,9 +1153,11 @@ __global__ void __launch_bounds__(128) dense_importance_kernel(const __grid_cons
             }
         }
     }
-    ok = !s_abort;
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 256);
+    }
 }
 
 template <int D, int NT>
@@ -1156,9 +1236,9 @@ int launch_dense(ScoreParams &p, const CUtensorMap &tm, cudaStream_t st) {
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_stats_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_STATS));
     AIRCACHE_CUDA_TRY(cudaFuncSetAttribute(dense_importance_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            C::SMEM_IMP));
-    dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), 128, C::SMEM_STATS, st>>>(tm, p);
+    dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), kDenseThreads, C::SMEM_STATS, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
-    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)p.n_lb), 128,
+    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)p.n_lb), kDenseThreads,
                                  C::SMEM_IMP, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
     return AIRCACHE_OK;
