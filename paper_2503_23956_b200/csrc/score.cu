@@ -536,8 +536,11 @@ __global__ void __launch_bounds__(128, 5) onepass_kernel(ScoreParams p) {
     const uint16_t *k_g = p.k + (int64_t)l * p.s_layer + (int64_t)b * p.s_batch + (int64_t)g * p.s_head;
     const int key0 = c * KB, key1 = min(p.Nv, key0 + KB);
     const int wk0 = key0 + warp * tpw * 16, wk1 = min(key1, wk0 + tpw * 16);
-    // the warp's whole key range is asked into L2 first: HBM latency runs beside the query staging
-    for (int i = lane; i < (wk1 - wk0) * (D * 2 / 128); i += 32)
+    // the warp's first two tiles are asked into L2 now (HBM latency runs beside the query staging), every later
+    // tile two tiles before its turn.  (Asking for the whole chunk at once measured 15 % slower: the burst
+    // queues in front of the loads that are waited for.)
+    constexpr int kAhead = 2 * 16;
+    for (int i = lane; i < min(wk1 - wk0, kAhead) * (D * 2 / 128); i += 32)
         prefetch_l2(k_g + (int64_t)(wk0 + i / (D * 2 / 128)) * p.s_token + (i % (D * 2 / 128)) * 64);
 
     auto fetch = [&](KeyFrag<D> &dst, int kt) {
@@ -599,6 +602,10 @@ __global__ void __launch_bounds__(128, 5) onepass_kernel(ScoreParams p) {
             const int ka = kt + gid, kb = kt + gid + 8;
             const bool va = ka < wk1, vb = kb < wk1;
             if (kt + 16 < wk1) fetch(f_next, kt + 16);
+            if (kt + kAhead < wk1 && lane < 16 * (D * 2 / 128)) {   // one 128-byte line per lane: 16 rows x d channels
+                const int kp = min(kt + kAhead + lane / (D * 2 / 128), wk1 - 1);
+                prefetch_l2(k_g + (int64_t)kp * p.s_token + (lane % (D * 2 / 128)) * 64);
+            }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 if (nt < nt_used) {
