@@ -98,8 +98,9 @@ inline int score_chunks(int n_visual, int64_t groups) {
 }
 
 // One-pass scoring (both passes of Eq. 7 in one block, logits kept on chip between them): a block covers 1024
-// keys of a KV group with up to 8 elite rows, 512 keys otherwise; the grid is laid out for 512.
-constexpr int kOnePassMinKeys = 512;
+// keys of a KV group with up to 8 elite rows, 512 keys otherwise, and as few as 256 in calls over few groups;
+// the workspace is laid out for 256.
+constexpr int kOnePassMinKeys = 256;
 constexpr int kOnePassMaxKeys = 1024;
 inline int onepass_chunks(int n_visual) { return (n_visual + kOnePassMinKeys - 1) / kOnePassMinKeys; }
 

@@ -43,7 +43,8 @@ struct ScoreParams {
     uint32_t *dispatch;     // one-pass scoring: blocks started so far
     float *imp_part;        // one-pass scoring: [L*B*Hkv][Nv] importance of one KV group
     uint16_t *q_block;      // one-pass scoring: [L*B*Hkv][16][d] the first 16 elite query rows, gathered
-    int op_chunks;
+    int op_chunks;      // numbers (blocks) per KV group in the one-pass grid
+    int op_tile_cap;    // most 16-key tiles a warp of the one-pass kernel takes: 16, or fewer when the call is small
     int L, B, Hq, Hkv, G, d, Nv, Nt, W;
     int lb0, n_lb;   // the launch covers regions lb0 .. lb0 + n_lb - 1 (a range of layers)
     int per_head;    // scores are kept apart per KV group: [L,B,Hkv,Nv], Eq. 8 averaged over the group's heads only
@@ -503,8 +504,8 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *ptr) {
     return v;
 }
 
-__device__ __forceinline__ int onepass_tiles(int n_rows) {   // 16-key tiles per warp
-    return n_rows <= 8 ? 16 : 8;
+__device__ __forceinline__ int onepass_tiles(int n_rows, int cap) {   // 16-key tiles per warp
+    return min(n_rows <= 8 ? 16 : 8, cap);
 }
 
 template <int D>
@@ -528,7 +529,7 @@ __global__ void __launch_bounds__(128, 5) onepass_kernel(ScoreParams p) {
     const int grp = p.lb0 * p.Hkv + gi;
     const int g = grp % p.Hkv, lb = grp / p.Hkv, l = lb / p.B, b = lb % p.B;
     const int n_rows = p.row_count[grp];
-    const int tpw = onepass_tiles(n_rows);
+    const int tpw = onepass_tiles(n_rows, p.op_tile_cap);
     const int KB = 64 * tpw;
     const int chunks_g = (p.Nv + KB - 1) / KB;
     if (c >= chunks_g) return;
@@ -1272,7 +1273,20 @@ int launch_score(const aircache_shape_t *s, const aircache_full_t *f, const void
     p.dispatch = ws_ptr<uint32_t>(ws, w.dispatch);
     p.imp_part = ws_ptr<float>(ws, w.imp_part);
     p.q_block = ws_ptr<uint16_t>(ws, w.q_block);
-    p.op_chunks = onepass_chunks(s->n_visual);
+    // A call over few KV groups (a layer at a time, a single short sequence) would leave SMs idle with 512- and
+    // 1024-key blocks: while the blocks would fill less than half of the GPU, they take half the tiles per warp,
+    // down to 256 keys per block (config 4 a layer at a time: 41 -> 33 us per layer).
+    {
+        const int resident = s->head_dim == 64 ? onepass_resident_blocks<64>() : onepass_resident_blocks<128>();
+        const int64_t groups = (int64_t)layer_count * s->batch * s->n_kv_heads;
+        auto numbers_per_group = [&](int cap) { const int k = 64 * (cap < 8 ? cap : 8); return (s->n_visual + k - 1) / k; };
+        p.op_tile_cap = 16;
+        while (p.op_tile_cap > 4 &&
+               groups * ((s->n_visual + 64 * p.op_tile_cap - 1) / (64 * p.op_tile_cap)) * 2 < (int64_t)resident &&
+               (int64_t)numbers_per_group(p.op_tile_cap / 2) * 2 <= resident)
+            p.op_tile_cap >>= 1;
+        p.op_chunks = numbers_per_group(p.op_tile_cap);
+    }
     p.L = s->n_layers; p.B = s->batch; p.Hq = s->n_q_heads; p.Hkv = s->n_kv_heads;
     p.G = s->n_q_heads / s->n_kv_heads; p.d = s->head_dim; p.Nv = s->n_visual; p.Nt = s->n_text; p.W = s->window;
     p.per_head = s->per_kv_head;
