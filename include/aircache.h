@@ -346,16 +346,18 @@ int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes);
  * queries, runs score -> budget -> compact -> n_steps x decode_attn on the
  * stream, downloads the results and synchronises.  Every device buffer is still
  * the caller's (no device memory is allocated inside).  K is uploaded whole
- * (the scoring passes read all of it, twice).  V is only ever read where a row
+ * (scoring reads all of it).  V is only ever read where a row
  * survives: if h_full->v is page-locked host memory that the GPU can address
  * (cudaHostAlloc / cudaHostRegister; aircache_host_range_is_mapped() tells),
  * compaction reads the kept and the text rows of V from it in place and
- * d_full_v stays untouched; otherwise V is uploaded whole like K.  The outputs of the
- * decode rounds are copied back in groups of 16 rounds on a second stream that
- * the call creates and destroys, so that the download overlaps the later rounds;
- * on return every copy has completed.  The call clears the workspace's status
+ * d_full_v stays untouched; otherwise V is uploaded whole like K.  The decode
+ * queries are uploaded in groups of 16 rounds on a stream of their own, behind
+ * the caches and beside the compression and the earlier rounds, and the outputs
+ * of the decode rounds are copied back in groups of 16 rounds on another stream,
+ * beside the later rounds (the call creates and destroys both streams); on
+ * return every copy has completed.  The call clears the workspace's status
  * words itself.  If a copy or a launch fails after the first copy has been
- * enqueued, the call still drains both streams before it returns the error, so
+ * enqueued, the call still drains all its streams before it returns the error, so
  * the host buffers are never touched after the return; the device buffers then
  * hold partial results.
  *   h_full       HOST view of the full cache (strides as in aircache_full_t)

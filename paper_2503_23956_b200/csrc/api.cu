@@ -3,6 +3,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <vector>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -358,14 +360,19 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
 
     // From here on work is in flight on the stream (and later on the copy stream) that reads and writes the
     // caller's host buffers: whatever happens, the call returns only after both streams have drained.
+    constexpr int32_t kCopyEvery = 16;   // decode rounds per upload of queries and per download of outputs
     struct CopySide {
-        cudaStream_t main = nullptr, stream = nullptr;
+        cudaStream_t main = nullptr, stream = nullptr, up = nullptr;
         cudaEvent_t event = nullptr;
+        std::vector<cudaEvent_t> arrived;   // one per block of kCopyEvery rounds: its queries are on the device
         ~CopySide() {
+            if (up) cudaStreamSynchronize(up);
             if (stream) cudaStreamSynchronize(stream);
             cudaStreamSynchronize(main);
             if (event) cudaEventDestroy(event);
+            for (cudaEvent_t e : arrived) cudaEventDestroy(e);
             if (stream) cudaStreamDestroy(stream);
+            if (up) cudaStreamDestroy(up);
         }
     } side;
     side.main = st;
@@ -373,9 +380,26 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
     if (!v_in_place)
         AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_full_v, h_full->v, full_elems * 2, cudaMemcpyHostToDevice, st));
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_q_window, h_q_window, qw_bytes, cudaMemcpyHostToDevice, st));
-    if (n_steps > 0)
-        AIRCACHE_CUDA_TRY(cudaMemcpyAsync(d_q_steps, h_q_steps, (int64_t)n_steps * q_elems * 2,
-                                          cudaMemcpyHostToDevice, st));
+    // The decode queries are needed round by round only: a third stream uploads them, kCopyEvery rounds at a
+    // time, behind the caches (which the compression is waiting for) and beside the compression and the
+    // earlier rounds; a round waits for the event of its block.
+    if (n_steps > 0) {
+        AIRCACHE_CUDA_TRY(cudaStreamCreateWithFlags(&side.stream, cudaStreamNonBlocking));
+        AIRCACHE_CUDA_TRY(cudaStreamCreateWithFlags(&side.up, cudaStreamNonBlocking));
+        AIRCACHE_CUDA_TRY(cudaEventCreateWithFlags(&side.event, cudaEventDisableTiming));
+        AIRCACHE_CUDA_TRY(cudaEventRecord(side.event, st));
+        AIRCACHE_CUDA_TRY(cudaStreamWaitEvent(side.up, side.event, 0));
+        for (int32_t first = 0; first < n_steps; first += kCopyEvery) {
+            const int32_t n = n_steps - first < kCopyEvery ? n_steps - first : kCopyEvery;
+            AIRCACHE_CUDA_TRY(cudaMemcpyAsync((char *)d_q_steps + (int64_t)first * q_elems * 2,
+                                              (const char *)h_q_steps + (int64_t)first * q_elems * 2,
+                                              (int64_t)n * q_elems * 2, cudaMemcpyHostToDevice, side.up));
+            cudaEvent_t e = nullptr;
+            AIRCACHE_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            side.arrived.push_back(e);
+            AIRCACHE_CUDA_TRY(cudaEventRecord(e, side.up));
+        }
+    }
     if ((rc = aircache_reset_status(workspace, workspace_bytes, st))) return rc;
     if ((rc = aircache_score(shape, &d_full, d_q_window, alpha, d_scores, nullptr, workspace, workspace_bytes, st)))
         return rc;
@@ -387,12 +411,8 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
         return rc;
     // The results go back to the host while later rounds still run: a second stream copies every
     // kCopyEvery rounds' outputs as soon as the round that wrote the last of them has finished.
-    constexpr int32_t kCopyEvery = 16;
-    if (n_steps > 0) {
-        AIRCACHE_CUDA_TRY(cudaStreamCreateWithFlags(&side.stream, cudaStreamNonBlocking));
-        AIRCACHE_CUDA_TRY(cudaEventCreateWithFlags(&side.event, cudaEventDisableTiming));
-    }
     for (int32_t i = 0; i < n_steps; ++i) {
+        if (i % kCopyEvery == 0) AIRCACHE_CUDA_TRY(cudaStreamWaitEvent(st, side.arrived[i / kCopyEvery], 0));
         const char *q = (const char *)d_q_steps + (int64_t)i * q_elems * 2;
         if ((rc = aircache_decode_attn(shape, d_cache, q, d_out + (int64_t)i * q_elems, workspace,
                                        workspace_bytes, st)))
@@ -407,7 +427,10 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
         }
     }
     AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_budgets, d_budgets, n_cells(shape) * 4, cudaMemcpyDeviceToHost, st));
-    if (n_steps > 0) AIRCACHE_CUDA_TRY(cudaStreamSynchronize(side.stream));
+    if (n_steps > 0) {
+        AIRCACHE_CUDA_TRY(cudaStreamSynchronize(side.up));
+        AIRCACHE_CUDA_TRY(cudaStreamSynchronize(side.stream));
+    }
     AIRCACHE_CUDA_TRY(cudaStreamSynchronize(st));
     return AIRCACHE_OK;
 }
