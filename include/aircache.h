@@ -34,10 +34,11 @@
  *             issues many copies and launches, is the exception: see there).
  *             No exception crosses the ABI.
  * Threads.    The library keeps no mutable global state apart from a per-thread
- *             copy of the last CUDA error code and the device address of the
- *             built-in array of aircache_decode_attn_static (looked up once per
- *             device, under a lock); calls that share a workspace must be ordered
- *             on one stream.
+ *             copy of the last CUDA error code, the device address of the
+ *             built-in array of aircache_decode_attn_static and the number of
+ *             blocks of the scoring kernel a device holds at once (each looked
+ *             up once per device, under a lock); calls that share a workspace
+ *             must be ordered on one stream.
  * Determinism. Same inputs give the same output bits on every run.
  */
 #ifndef AIRCACHE_H
@@ -174,6 +175,12 @@ int64_t aircache_workspace_bytes(const aircache_shape_t *shape);
  *   scores      fp32 [L, B, Nv]        output I_v
  *   elite_mask  u64  [L, B, Hq, ceil(W/64)]  output, candidate w is elite <=> bit w % 64 of word w / 64 is
  *                                      set (one word per head up to W = 64, two beyond); may be NULL
+ * The blocks of the scoring kernel that share a KV group wait for one another
+ * (a bounded wait; safe because the library only lets them when at most half of
+ * the blocks the GPU holds at once are involved).  If other work keeps most of
+ * the GPU busy for the whole wait (a quarter of a second), the wait gives up,
+ * the scores are incomplete and aircache_check_status() reports
+ * AIRCACHE_ERR_TIMEOUT.
  */
 int aircache_score(const aircache_shape_t *shape, const aircache_full_t *full, const void *q_window,
                    float alpha, float *scores, uint64_t *elite_mask, void *workspace, int64_t workspace_bytes,

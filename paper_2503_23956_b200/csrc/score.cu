@@ -20,6 +20,8 @@
 // per CTA, so staging it in shared memory would only add a round trip.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -740,13 +742,16 @@ __global__ void __launch_bounds__(256) group_sum_kernel(ScoreParams p) {
     p.scores[(int64_t)lb * p.Nv + i] = v;
 }
 
-// Blocks of the one-pass kernel the device holds at once (0 if the kernel cannot run); asked once per device.
+// Blocks of the one-pass kernel the device holds at once (0 if the kernel cannot run); asked once per device,
+// under a lock.
 template <int D>
 int onepass_resident_blocks() {
+    static std::mutex lock;
     static int cached[64];
     static bool have[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    std::lock_guard<std::mutex> guard(lock);
     if (!have[dev]) {
         int per_sm = 0, sms = 0;
         if (cudaFuncSetAttribute(onepass_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768) != cudaSuccess ||
