@@ -125,6 +125,33 @@ def test_score_parity_sequence_longer_than_the_one_pass_kernel_takes(oracle):
     assert err <= TOL, err
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_score_parity_random_mid_size_shapes(oracle, seed):
+    """Seeded random shapes with thousands of visual tokens (several key chunks per KV group, ragged tails), head
+    layouts from 1 to 8 KV heads and 1 to 16 heads per group, windows up to the whole text, thresholds that give
+    from one to over a hundred elite rows per group, per layer and per KV head: masks equal, scores within the
+    tolerance."""
+    rng = np.random.default_rng(1000 + seed)
+    hkv, g, d = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4, 7, 8, 16])), int(rng.choice([64, 128]))
+    L, B = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    nv, nt = int(rng.integers(300, 9000)), int(rng.integers(16, 130))
+    W = int(rng.integers(1, min(nt, 128) + 1))
+    alpha = float(rng.choice([0.9, 0.9, 0.5, 0.1, 1e-3, 0.99]))
+    per_kv_head = seed % 2
+    wl = small(f"mid{seed}", L=L, Hq=hkv * g, Hkv=hkv, d=d, B=B, Nv=nv, Nt=nt, W=W, alpha=alpha)
+    k, v, qw = cpu_inputs(wl)
+    dm = oracle_dims(oracle, wl)
+    fn = oracle.score_groups if per_kv_head else oracle.score
+    sc = fn(dm, u16(logical(k)), u16(qw), wl.scale, alpha)
+    gp = GpuPath(wl, device=DEV, per_kv_head=per_kv_head)
+    gp.set_full(logical(k.to(DEV)), logical(v.to(DEV)))
+    gp.score(qw.to(DEV), alpha=alpha)
+    assert gp.status() == 0
+    assert np.array_equal(gp.mask.cpu().numpy().view(np.uint64).reshape(-1), sc["elite_mask"].reshape(-1)), wl
+    err = rel_elem_err(gp.scores.cpu().numpy().reshape(-1), sc["scores"].reshape(-1))
+    assert err <= TOL, (wl, err)
+
+
 @pytest.mark.parametrize("case", ["kv2", "s7b", "g16", "w128"])
 def test_score_parity_many_elite_rows_below_the_dense_threshold(oracle, case):
     """A small but non-zero threshold makes almost every candidate elite (hundreds of rows per KV group on the
