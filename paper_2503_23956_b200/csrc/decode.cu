@@ -1202,7 +1202,7 @@ int launch_decode_d(const aircache_shape_t *s, const aircache_ragged_t *c, Decod
     int sms = 0;
     int rc = sm_count(&sms);
     if (rc) return rc;
-    if (hkv > 1 && p.n_regions * hkv <= (sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas)) {
+    if (p.n_regions * hkv <= (sms < kMaxDecodeCtas ? sms : kMaxDecodeCtas)) {   // also with one KV head: an item is a region
         p.hs = hkv;
         p.n_regions *= hkv;
         p.Hq = p.G;
