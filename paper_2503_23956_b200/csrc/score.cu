@@ -7,17 +7,20 @@
 //                      the Eq. 5 decision does not depend on a summation order), the elite set of each
 //                      query head, the table of elite rows (head, window slot) of the KV group, and each
 //                      row's softmax statistics over the text keys it may see (elite, causal).
-//   stats_kernel       Eq. 7 pass one: Q_tk K_v^T on tensor cores (keys on the M axis, elite rows on N),
-//                      running (max, sum of exp2) of every elite row over one chunk of visual keys.  The CTA
+//                      It also leaves a gathered copy of the group's first 16 elite query rows.
+//   onepass_kernel     Eq. 7 and Eq. 8 with one read of the visual keys: Q_tk K_v^T on tensor cores (keys on
+//   + group_sum_kernel the M axis, elite rows on N), a chunk's logits kept in shared memory between the
+//                      statistics and the probabilities; see the comment at the kernel.  The normal path.
+//   stats_kernel       the same in two passes, for sequences too long for the one-pass kernel.  Pass one:
+//   + importance_kernel running (max, sum of exp2) of every elite row over one chunk of visual keys; the CTA
 //                      that finishes a KV group last (ticket) merges the chunks and the text statistics
-//                      into one (max, weight / normaliser) pair per row.
-//   importance_kernel  Eq. 7 pass two + Eq. 8: recomputes the same tiles (keys now come from L2 when the
-//                      cache is small enough), turns logits into probabilities and sums the rows of all
-//                      heads per key with weight 1 / (|E_h| Hq).  KV heads are visited in ascending order
-//                      by one thread per key, so the sum has a fixed order.
+//                      into one (max, weight / normaliser) pair per row.  Pass two recomputes the same
+//                      tiles, turns logits into probabilities and sums the rows of all heads per key with
+//                      weight 1 / (|E_h| Hq), KV heads in ascending order by one thread per key.
+//   dense_*_kernel     alpha = 0 (every window query elite): both passes on tcgen05, see there.
 //
-// Both passes read the keys straight from global memory into MMA fragments: every key byte is used once
-// per CTA, so staging it in shared memory would only add a round trip.
+// The mma.sync kernels read the keys straight from global memory into MMA fragments: every key byte is used
+// once per CTA, so staging it in shared memory would only add a round trip.
 #include <math.h>
 
 #include <mutex>
