@@ -798,7 +798,6 @@ struct DenseCfg {
     static constexpr int TILE_BYTES = KSUB * SUB_BYTES;
     static constexpr int NST = 2;                   // key tiles in flight (two CTAs share an SM)
     static constexpr int SMEM_STATS = 1024 + (NST + 1) * TILE_BYTES + 256;
-    static constexpr int KT = 4;                    // key tiles per CTA of the importance pass
     static constexpr int SMEM_IMP = 1024 + (NST + 1) * TILE_BYTES + 128 * 8 + 256;
 };
 
@@ -887,13 +886,30 @@ struct DensePipe {
 
 // The driver thread's part for n_tiles key tiles starting at key0: `base` tiles went through the pipe before.
 // a_is_query: the query block is the MMA's A operand (rows on M, pass one), else the key tile is (keys on M).
+// The first key tiles of a block of work, issued by the driver thread while the other warps stage the query
+// block: returns how many loads are under way (the stages are free: the previous block's MMAs have completed).
+template <int D>
+__device__ __forceinline__ int dense_first_loads(const DensePipe<D> &pp, const CUtensorMap *tm, const ScoreParams &p,
+                                                 uint8_t *s_k, uint32_t base, int n_tiles, int key0, int g, int b, int l,
+                                                 volatile int *s_abort, uint32_t code) {
+    using C = DenseCfg<D>;
+    int loaded = 0;
+    while (loaded < n_tiles && loaded < C::NST) {
+        const uint32_t il = base + loaded, ls = il % C::NST;
+        if (!mbar_wait(pp.empty[ls], ((il / C::NST) & 1) ^ 1, s_abort, p.status, code)) break;
+        load_key_tile<D>(smem_u32(s_k + ls * C::TILE_BYTES), tm, p, key0 + loaded * 128, g, b, l, pp.full[ls]);
+        ++loaded;
+    }
+    return loaded;
+}
+
 template <int D, bool A_IS_QUERY>
 __device__ __forceinline__ bool dense_drive(const DensePipe<D> &pp, const CUtensorMap *tm, const ScoreParams &p,
                                             uint32_t tmem, uint8_t *s_k, uint8_t *s_q, uint32_t base, int n_tiles,
-                                            int key0, int g, int b, int l, volatile int *s_abort, uint32_t code) {
+                                            int loaded, int key0, int g, int b, int l, volatile int *s_abort,
+                                            uint32_t code) {
     using C = DenseCfg<D>;
     bool ok = true;
-    int loaded = 0;
     for (int t = 0; t < n_tiles && ok; ++t) {
         while (ok && loaded < n_tiles && loaded < t + C::NST) {
             const uint32_t il = base + loaded, ls = il % C::NST;
@@ -956,11 +972,13 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
     for (int row0 = 0; row0 < n_rows; row0 += 128) {
         __syncthreads();   // the previous block's MMAs have completed (their logits were read): the query block is free
         if (s_abort) break;
+        int loaded = 0;
         if (tid < 128) stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
+        else if (tid == 128) loaded = dense_first_loads<D>(pp, &tm_k, p, s_k, base, n_tiles, key0, g, b, l, &s_abort, 4);
         __syncthreads();
         if (warp == 4) {
             if (lane == 0)
-                dense_drive<D, true>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, key0, g, b, l, &s_abort, 4);
+                dense_drive<D, true>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, loaded, key0, g, b, l, &s_abort, 4);
         } else {
             float m = kNegBig, z = 0.f;
             bool ok = true;
@@ -1059,11 +1077,12 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
     }
 }
 
-// Pass two, dense.  grid = (ceil(Nv / (128*KT)), L*B), 160 threads; an epilogue thread owns one key per tile.
+// Pass two, dense.  grid = (chunks, L*B*Hkv) like pass one, 160 threads; an epilogue thread owns one key per tile
+// and adds the weighted probabilities of the group's rows.  The group's sums go to its row of the per-group
+// buffer (group_sum_kernel adds the groups), or straight to the scores in per-KV-head mode.
 template <int D>
 __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     using C = DenseCfg<D>;
-    constexpr int KT = C::KT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *s_k = smem;                             // NST key tiles
@@ -1074,10 +1093,13 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int lb = p.lb0 + blockIdx.y;
+    const int grp = p.lb0 * p.Hkv + blockIdx.y;
+    const int g = grp % p.Hkv, lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
-    const int key0 = blockIdx.x * 128 * KT;
-    const int n_tiles = min(KT, (p.Nv - key0 + 127) / 128);
+    const int key0 = blockIdx.x * p.chunk_keys, key1 = min(p.Nv, key0 + p.chunk_keys);
+    const int n_tiles = key1 > key0 ? (key1 - key0 + 127) / 128 : 0;
+    const int n_rows = p.row_count[grp];
+    float *out = (p.per_head ? p.scores : p.imp_part) + (int64_t)grp * p.Nv;
 
     DensePipe<D> pp;
     pp.init(s_bar);
@@ -1092,82 +1114,67 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     uint32_t base = 0;
-    float imp[KT];
-#pragma unroll
-    for (int t = 0; t < KT; ++t) imp[t] = 0.f;
 
-    for (int g = 0; g < p.Hkv; ++g) {
-        const int grp = lb * p.Hkv + g;
-        const int n_rows = p.row_count[grp];
-        for (int row0 = 0; row0 < n_rows; row0 += 128) {
-            __syncthreads();   // the previous block's MMAs have completed: query block and statistics are free
-            if (s_abort) break;
-            if (tid < 128) {
-                stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
-                s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
-            }
-            __syncthreads();
-            if (warp == 4) {
-                if (lane == 0)
-                    dense_drive<D, false>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, key0, g, b, l, &s_abort, 10);
-            } else {
-                const int nch = (min(128, n_rows - row0) + 31) >> 5;   // chunks of 32 rows with a real row in them
-                // 32 rows of the thread's key: probabilities weighted and summed
-                auto chunk32 = [&](const uint32_t (&r)[32], int c0) {
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};   // interleaved partial sums: short dependent chains
+    for (int row0 = 0; row0 < n_rows; row0 += 128) {
+        __syncthreads();   // the previous block's MMAs have completed: query block and statistics are free
+        if (s_abort) break;
+        int loaded = 0;
+        if (tid < 128) {
+            stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
+            s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
+        } else if (tid == 128) {
+            loaded = dense_first_loads<D>(pp, &tm_k, p, s_k, base, n_tiles, key0, g, b, l, &s_abort, 10);
+        }
+        __syncthreads();
+        if (warp == 4) {
+            if (lane == 0)
+                dense_drive<D, false>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, loaded, key0, g, b, l, &s_abort, 10);
+        } else {
+            const int nch = (min(128, n_rows - row0) + 31) >> 5;   // chunks of 32 rows with a real row in them
+            // 32 rows of the thread's key: probabilities weighted and summed
+            auto chunk32 = [&](const uint32_t (&r)[32], int c0) {
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};   // interleaved partial sums: short dependent chains
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float2 sj = s_stat[c0 + j];
-                        acc[j & 3] = fmaf(fast_exp2(fmaf(__uint_as_float(r[j]), p.sl2, -sj.x)), sj.y, acc[j & 3]);
-                    }
-                    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
-                };
-#pragma unroll
-                for (int t = 0; t < KT; ++t) {
-                    if (t >= n_tiles) break;
-                    const uint32_t it = base + t, a = it & 1;
-                    if (!mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 12)) break;
-                    tc_fence_after();
-                    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
-                    uint32_t r0[32], r1[32];
-                    float acc = 0.f;
-                    tmem_ld32_issue(taddr, r0);
-                    tmem_ld_wait(r0);
-                    if (nch > 1) tmem_ld32_issue(taddr + 32, r1);
-                    acc += chunk32(r0, 0);
-                    if (nch > 1) {
-                        tmem_ld_wait(r1);
-                        if (nch > 2) tmem_ld32_issue(taddr + 64, r0);
-                        acc += chunk32(r1, 32);
-                        if (nch > 2) {
-                            tmem_ld_wait(r0);
-                            if (nch > 3) tmem_ld32_issue(taddr + 96, r1);
-                            acc += chunk32(r0, 64);
-                            if (nch > 3) {
-                                tmem_ld_wait(r1);
-                                acc += chunk32(r1, 96);
-                            }
+                for (int j = 0; j < 32; ++j) {
+                    const float2 sj = s_stat[c0 + j];
+                    acc[j & 3] = fmaf(fast_exp2(fmaf(__uint_as_float(r[j]), p.sl2, -sj.x)), sj.y, acc[j & 3]);
+                }
+                return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            };
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t it = base + t, a = it & 1;
+                if (!mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 12)) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
+                uint32_t r0[32], r1[32];
+                float acc = 0.f;
+                tmem_ld32_issue(taddr, r0);
+                tmem_ld_wait(r0);
+                if (nch > 1) tmem_ld32_issue(taddr + 32, r1);
+                acc += chunk32(r0, 0);
+                if (nch > 1) {
+                    tmem_ld_wait(r1);
+                    if (nch > 2) tmem_ld32_issue(taddr + 64, r0);
+                    acc += chunk32(r1, 32);
+                    if (nch > 2) {
+                        tmem_ld_wait(r0);
+                        if (nch > 3) tmem_ld32_issue(taddr + 96, r1);
+                        acc += chunk32(r0, 64);
+                        if (nch > 3) {
+                            tmem_ld_wait(r1);
+                            acc += chunk32(r1, 96);
                         }
                     }
-                    imp[t] += acc;
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(pp.acc_empty[a]);
                 }
-            }
-            base += n_tiles;
-        }
-        if (s_abort) break;
-        if (tid < 128 && (p.per_head || g == p.Hkv - 1)) {
-            // the keys' scores are complete: of this KV group alone, or summed over all of them
-            float *out = p.scores + (p.per_head ? (int64_t)grp : (int64_t)lb) * p.Nv;
-#pragma unroll
-            for (int t = 0; t < KT; ++t) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pp.acc_empty[a]);
+                // the thread's key of this tile: first row block writes, later ones add (same thread every time)
                 const int key = key0 + t * 128 + tid;
-                if (t < n_tiles && key < p.Nv) out[key] = imp[t];
-                imp[t] = 0.f;
+                if (key < key1) out[key] = row0 == 0 ? acc : out[key] + acc;
             }
         }
+        base += n_tiles;
     }
     __syncthreads();
     if (warp == 4) {
@@ -1254,9 +1261,12 @@ int launch_dense(ScoreParams &p, const CUtensorMap &tm, cudaStream_t st) {
                                            C::SMEM_IMP));
     dense_stats_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), kDenseThreads, C::SMEM_STATS, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
-    dense_importance_kernel<D><<<dim3((p.Nv + 128 * C::KT - 1) / (128 * C::KT), (unsigned)p.n_lb), kDenseThreads,
-                                 C::SMEM_IMP, st>>>(tm, p);
+    dense_importance_kernel<D><<<dim3(p.chunks, (unsigned)((int64_t)p.n_lb * p.Hkv)), kDenseThreads, C::SMEM_IMP, st>>>(tm, p);
     AIRCACHE_LAUNCH_CHECK();
+    if (!p.per_head) {
+        group_sum_kernel<<<dim3((p.Nv + 255) / 256, (unsigned)p.n_lb), 256, 0, st>>>(p);
+        AIRCACHE_LAUNCH_CHECK();
+    }
     return AIRCACHE_OK;
 }
 
