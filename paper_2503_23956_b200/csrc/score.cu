@@ -861,13 +861,15 @@ __device__ __forceinline__ void load_key_tile(uint32_t dst, const CUtensorMap *t
         tma_load_5d(dst + sub * DenseCfg<D>::SUB_BYTES, tm, sub * 64, c[1], c[2], c[3], c[4], bar);
 }
 
-// Both dense kernels are warp-specialised: warps 0-3 own one accumulator row per thread (a tensor-memory lane)
-// and run the exponent arithmetic; one thread of warp 4 drives the copies and the tensor core.  Key tiles cycle
-// through NST shared-memory stages (full: TMA landed; empty: the MMAs that read the stage have completed, by
-// tcgen05.commit), accumulators through two halves of 256 tensor-memory columns (acc_full by tcgen05.commit,
-// acc_empty by one arrival per epilogue warp): the MMAs of tile t+1 run while tile t's logits are read back
-// and exponentiated.  Parities follow from running tile counts.  Every wait is bounded.
-constexpr int kDenseThreads = 160;
+// Both dense kernels are warp-specialised: two sets of four epilogue warps (warps 0-3 and 4-7; a thread owns one
+// accumulator row, a tensor-memory lane) run the exponent arithmetic, one thread of warp 8 drives the copies
+// and the tensor core.  Key tiles cycle through NST shared-memory stages (full: TMA landed; empty: the MMAs
+// that read the stage have completed, by tcgen05.commit), accumulators through two halves of 256 tensor-memory
+// columns (acc_full by tcgen05.commit, acc_empty by one arrival per warp of the set that read it).  Each set
+// takes the tiles of one accumulator, so two tiles' logits are read back and exponentiated at a time while the
+// MMAs of the next run.  Parities follow from running tile counts.  Every wait is bounded.
+constexpr int kDenseThreads = 288;
+constexpr int kDenseDriverWarp = 8;
 
 template <int D>
 struct DensePipe {
@@ -935,7 +937,7 @@ __device__ __forceinline__ bool dense_drive(const DensePipe<D> &pp, const CUtens
 
 // Pass one, dense.  grid = (chunks, L*B*Hkv), 160 threads.
 template <int D>
-__global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+__global__ void __launch_bounds__(kDenseThreads, 2) dense_stats_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     using C = DenseCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -946,6 +948,8 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
     __shared__ int s_abort, s_is_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int set = warp >> 2, row = (warp & 3) * 32 + lane;   // epilogue set and accumulator row (warps 0-7)
+    __shared__ float2 s_mz[128];                               // the second set's (max, sum) of every row
     const int grp = p.lb0 * p.Hkv + blockIdx.y;
     const int g = grp % p.Hkv, lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
@@ -962,7 +966,7 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
         s_abort = 0;
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 4) tmem_alloc(smem_u32(&s_tmem), 256);
+    if (warp == kDenseDriverWarp) tmem_alloc(smem_u32(&s_tmem), 256);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -974,9 +978,11 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
         if (s_abort) break;
         int loaded = 0;
         if (tid < 128) stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
-        else if (tid == 128) loaded = dense_first_loads<D>(pp, &tm_k, p, s_k, base, n_tiles, key0, g, b, l, &s_abort, 4);
+        else if (tid == kDenseDriverWarp * 32) loaded = dense_first_loads<D>(pp, &tm_k, p, s_k, base, n_tiles, key0, g, b, l, &s_abort, 4);
         __syncthreads();
-        if (warp == 4) {
+        float m_mine = kNegBig, z_mine = 0.f;
+        bool ok_mine = true;
+        if (warp == kDenseDriverWarp) {
             if (lane == 0)
                 dense_drive<D, true>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, loaded, key0, g, b, l, &s_abort, 4);
         } else {
@@ -1011,12 +1017,13 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
                 z = z * fast_exp2(m - mn) + sum;
                 m = mn;
             };
-            for (int t = 0; t < n_tiles; ++t) {
+            // this set's tiles: those whose accumulator (running tile count, low bit) is the set's
+            for (int t = (set - (int)base) & 1; t < n_tiles; t += 2) {
                 const uint32_t it = base + t, a = it & 1;
                 ok = mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 6);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
+                const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + a * 128;
                 const int kbase = key0 + t * 128;
                 uint32_t r0[32], r1[32];
                 tmem_ld32_issue(taddr, r0);
@@ -1036,13 +1043,19 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
                 if (lane == 0) mbar_arrive(pp.acc_empty[a]);
                 chunk32(r1, kbase + 96);
             }
-            if (ok && row0 + tid < n_rows) __stcg(out + row0 + tid, make_float2(m, z));
+            if (set == 1) s_mz[row] = make_float2(m, z);
+            m_mine = m; z_mine = z; ok_mine = ok;
+        }
+        __syncthreads();   // the second set's half of every row's statistics is in shared memory
+        if (warp < 4 && ok_mine) {
+            merge_stats(m_mine, z_mine, s_mz[row].x, s_mz[row].y);
+            if (row0 + row < n_rows) __stcg(out + row0 + row, make_float2(m_mine, z_mine));
         }
         base += n_tiles;
     }
     __syncthreads();
     const bool ok = !s_abort;
-    if (warp == 4) {
+    if (warp == kDenseDriverWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, 256);
     }
@@ -1056,7 +1069,7 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
         if (s_is_last) __threadfence();
     }
     __syncthreads();
-    if (!s_is_last || warp >= 4) return;
+    if (!s_is_last || warp >= 4) return;   // four warps merge
     for (int r = warp; r < n_rows; r += 4) {
         float mm = kNegBig, zz = 0.f;
         if (lane == 0) {
@@ -1081,7 +1094,7 @@ __global__ void __launch_bounds__(kDenseThreads) dense_stats_kernel(const __grid
 // and adds the weighted probabilities of the group's rows.  The group's sums go to its row of the per-group
 // buffer (group_sum_kernel adds the groups), or straight to the scores in per-KV-head mode.
 template <int D>
-__global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
+__global__ void __launch_bounds__(kDenseThreads, 2) dense_importance_kernel(const __grid_constant__ CUtensorMap tm_k, ScoreParams p) {
     using C = DenseCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1093,6 +1106,7 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int set = warp >> 2, row = (warp & 3) * 32 + lane;   // epilogue set and accumulator row (warps 0-7)
     const int grp = p.lb0 * p.Hkv + blockIdx.y;
     const int g = grp % p.Hkv, lb = grp / p.Hkv;
     const int l = lb / p.B, b = lb % p.B;
@@ -1108,7 +1122,7 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
         s_abort = 0;
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
     }
-    if (warp == 4) tmem_alloc(smem_u32(&s_tmem), 256);
+    if (warp == kDenseDriverWarp) tmem_alloc(smem_u32(&s_tmem), 256);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -1122,11 +1136,11 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
         if (tid < 128) {
             stage_queries_sw128<D>(s_q, p, grp, lb, g, row0, n_rows);
             s_stat[tid] = row0 + tid < n_rows ? p.row_final[(int64_t)grp * p.cap + row0 + tid] : make_float2(0.f, 0.f);
-        } else if (tid == 128) {
+        } else if (tid == kDenseDriverWarp * 32) {
             loaded = dense_first_loads<D>(pp, &tm_k, p, s_k, base, n_tiles, key0, g, b, l, &s_abort, 10);
         }
         __syncthreads();
-        if (warp == 4) {
+        if (warp == kDenseDriverWarp) {
             if (lane == 0)
                 dense_drive<D, false>(pp, &tm_k, p, tmem, s_k, s_q, base, n_tiles, loaded, key0, g, b, l, &s_abort, 10);
         } else {
@@ -1141,11 +1155,12 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
                 }
                 return (acc[0] + acc[1]) + (acc[2] + acc[3]);
             };
-            for (int t = 0; t < n_tiles; ++t) {
+            // this set's tiles: those whose accumulator (running tile count, low bit) is the set's
+            for (int t = (set - (int)base) & 1; t < n_tiles; t += 2) {
                 const uint32_t it = base + t, a = it & 1;
                 if (!mbar_wait(pp.acc_full[a], (it >> 1) & 1, &s_abort, p.status, 12)) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + a * 128;
+                const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + a * 128;
                 uint32_t r0[32], r1[32];
                 float acc = 0.f;
                 tmem_ld32_issue(taddr, r0);
@@ -1170,14 +1185,14 @@ __global__ void __launch_bounds__(kDenseThreads) dense_importance_kernel(const _
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pp.acc_empty[a]);
                 // the thread's key of this tile: first row block writes, later ones add (same thread every time)
-                const int key = key0 + t * 128 + tid;
+                const int key = key0 + t * 128 + row;
                 if (key < key1) out[key] = row0 == 0 ? acc : out[key] + acc;
             }
         }
         base += n_tiles;
     }
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kDenseDriverWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, 256);
     }
