@@ -360,7 +360,7 @@ int aircache_host_range_is_mapped(const void *host_ptr, int64_t bytes);
  * d_full_v stays untouched; otherwise V is uploaded whole like K.  The decode
  * queries are uploaded in groups of 16 rounds on a stream of their own, behind
  * the caches and beside the compression and the earlier rounds, and the outputs
- * of the decode rounds are copied back in groups of 16 rounds on another stream,
+ * of the decode rounds are copied back in groups of 4 rounds on another stream,
  * beside the later rounds (the call creates and destroys both streams); on
  * return every copy has completed.  The call clears the workspace's status
  * words itself.  If a copy or a launch fails after the first copy has been

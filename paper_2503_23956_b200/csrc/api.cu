@@ -360,7 +360,8 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
 
     // From here on work is in flight on the stream (and later on the copy stream) that reads and writes the
     // caller's host buffers: whatever happens, the call returns only after both streams have drained.
-    constexpr int32_t kCopyEvery = 16;   // decode rounds per upload of queries and per download of outputs
+    constexpr int32_t kCopyEvery = 16;   // decode rounds per upload of queries
+    constexpr int32_t kDownEvery = 4;    // decode rounds per download of outputs (the last block's copy is the tail)
     struct CopySide {
         cudaStream_t main = nullptr, stream = nullptr, up = nullptr;
         cudaEvent_t event = nullptr;
@@ -410,15 +411,15 @@ int aircache_pipeline_host(const aircache_shape_t *shape, const aircache_full_t 
                                workspace_bytes, st)))
         return rc;
     // The results go back to the host while later rounds still run: a second stream copies every
-    // kCopyEvery rounds' outputs as soon as the round that wrote the last of them has finished.
+    // kDownEvery rounds' outputs as soon as the round that wrote the last of them has finished.
     for (int32_t i = 0; i < n_steps; ++i) {
         if (i % kCopyEvery == 0) AIRCACHE_CUDA_TRY(cudaStreamWaitEvent(st, side.arrived[i / kCopyEvery], 0));
         const char *q = (const char *)d_q_steps + (int64_t)i * q_elems * 2;
         if ((rc = aircache_decode_attn(shape, d_cache, q, d_out + (int64_t)i * q_elems, workspace,
                                        workspace_bytes, st)))
             return rc;
-        if ((i + 1) % kCopyEvery == 0 || i + 1 == n_steps) {
-            const int32_t first = i / kCopyEvery * kCopyEvery;
+        if ((i + 1) % kDownEvery == 0 || i + 1 == n_steps) {
+            const int32_t first = i / kDownEvery * kDownEvery;
             AIRCACHE_CUDA_TRY(cudaEventRecord(side.event, st));
             AIRCACHE_CUDA_TRY(cudaStreamWaitEvent(side.stream, side.event, 0));
             AIRCACHE_CUDA_TRY(cudaMemcpyAsync(h_out + (int64_t)first * q_elems, d_out + (int64_t)first * q_elems,
